@@ -1,0 +1,161 @@
+/*
+ * lbp.h -- C ABI of the LBP-WHT linear-layer backward library for NVIDIA B200
+ * (sm_100a).
+ *
+ * The library computes the backward pass of a linear layer y = x w^T the
+ * LBP-WHT way (Low-rank BackPropagation via Walsh-Hadamard Transformation,
+ * arXiv 2309.15275): x and g_y are projected onto r two-dimensional
+ * Walsh-Hadamard bases per k x k block of the token grid (Eq. 3, Eq. 6), the
+ * two gradient products run in that low-rank space (Eq. 4, Algorithm 1), and
+ * the low-rank input gradient is expanded back with the transposed bases
+ * (Eq. 5, Eq. 7).
+ *
+ * Conventions, valid for every entry point unless it says otherwise
+ *  - Tensor pointers (x, g_y, W, g_x, g_W, t, t_hat, ws) are DEVICE pointers
+ *    owned by the caller; they must be 16-byte aligned and C * element size
+ *    must be a multiple of 16 bytes.  The library never allocates or frees
+ *    device memory and keeps no per-call state.
+ *  - Basis lists, layer descriptors and every other pointer are HOST pointers,
+ *    read during the call and not retained.
+ *  - Layouts are dense, channels-last raster:
+ *        x   (B, H, W, Cin)     g_y (B, H, W, Cout)     g_x (B, H, W, Cin)
+ *        W, g_W (Cout, Cin) row-major (w in R^{Cy x Cx} of Eq. 1)
+ *        t_hat (B, H/k, W/k, r, C): coefficient q of a block follows the order
+ *        of the basis list.
+ *    Tokens are grouped into non-overlapping, origin-aligned k x k blocks of
+ *    the (H, W) grid; H and W must be multiples of k.
+ *  - Bases are orthonormal: the +-1 Walsh bases of Eq. 6-7 are scaled by 1/k
+ *    in the projection and by 1/k in the reverse projection, so that all k*k
+ *    bases reproduce exact backpropagation (Sec. 3, completeness).
+ *  - A basis (i, j) is the outer product of the Walsh rows with i sign changes
+ *    along H and j sign changes along W, 0 <= i, j < k (sequency order: a
+ *    smaller index is a lower frequency, Sec. 3.2).
+ *  - `stream` is a cudaStream_t passed as void*.  Device work is enqueued on
+ *    it and the call returns without synchronising.  Argument errors are
+ *    detected before anything is enqueued: on a non-zero return no output has
+ *    been touched.  Waits inside kernels are bounded; an expired wait is
+ *    reported through the status word in `ws` (lbp_poll_status).
+ *  - Every function returns an lbp_status (0 = LBP_OK) unless it returns a
+ *    size, a number or a string.
+ */
+#ifndef LBP_H_
+#define LBP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LBP_OK = 0,
+  LBP_ERR_NULL = 1,       /* a required pointer is NULL                         */
+  LBP_ERR_SHAPE = 2,      /* a dimension <= 0, or H % k != 0, or W % k != 0      */
+  LBP_ERR_BLOCK = 3,      /* k not in {4, 8, 16}                                */
+  LBP_ERR_BASIS = 4,      /* r < 1, r > k*k, index outside [0,k), duplicate pair */
+  LBP_ERR_DTYPE = 5,      /* unknown dtype, or a combination not supported      */
+  LBP_ERR_ALIGN = 6,      /* pointer or C * element size not 16-byte aligned    */
+  LBP_ERR_WORKSPACE = 7,  /* ws is NULL or smaller than lbp_workspace_bytes()   */
+  LBP_ERR_ARCH = 8,       /* current device is not compute capability 10.x      */
+  LBP_ERR_CUDA = 9,       /* a CUDA call failed; see lbp_last_cuda_error()      */
+  LBP_ERR_TIMEOUT = 10,   /* a bounded device-side wait expired                 */
+  LBP_ERR_CAPACITY = 11   /* output array too small (lbp_select_bases)          */
+} lbp_status;
+
+typedef enum { LBP_F32 = 0, LBP_BF16 = 1 } lbp_dtype;
+
+/* Basis-selection rules of Sec. 3.2.  LP_L1 and LP_Linf are Eq. 8 and Eq. 9
+ * with 0-based indices (i + j <= m-1, max(i,j) <= m-1; ranks m(m+1)/2 and m*m,
+ * the ranks the paper's tables print).  PREFIX-r keeps the first r pairs of the
+ * total order key(i,j) = (i+j, max(i,j), i), which lists every LP_L1 set as a
+ * prefix and defines ranks that are neither triangular nor square. */
+typedef enum { LBP_SEL_L1 = 0, LBP_SEL_LINF = 1, LBP_SEL_PREFIX = 2 } lbp_rule;
+
+typedef struct { int32_t i, j; } lbp_basis;   /* 0-based sequency indices    */
+
+typedef struct {
+  int32_t B, H, W;        /* batch and token grid                               */
+  int32_t Cin, Cout;      /* C_x and C_y of Eq. 1                               */
+  int32_t k;              /* WHT order = block edge, 4, 8 or 16                 */
+  int32_t dtype;          /* lbp_dtype of x, g_y, W, g_x                        */
+  int32_t gw_dtype;       /* lbp_dtype of g_W (LBP_F32 allowed with bf16 data)  */
+} lbp_layer;
+
+/* ---- host-only helpers (no device needed) ------------------------------- */
+
+/* Sec. 3.2, Eq. 8-9.  Writes the ordered basis list chosen by `rule` with
+ * parameter `param` (m for LP_L1 / LP_Linf, r for PREFIX) for order k into
+ * out[0..*r_out).  All rules list their pairs in the PREFIX total order.
+ * out: host array of `cap` entries.  LBP_ERR_CAPACITY if cap is too small
+ * (*r_out still receives the needed count), LBP_ERR_BLOCK / LBP_ERR_BASIS for
+ * a bad k / param. */
+int lbp_select_bases(int k, int rule, int param, lbp_basis* out, int cap, int* r_out);
+
+/* Eq. 6: the k*k x r matrix (B_{i1,j1} ... B_{ir,jr}) of +-1 entries, row
+ * u*k+v (raster position inside a block), column q.  P_out: host array of
+ * k*k*r int8, row-major.  Validates the list like every other call. */
+int lbp_basis_matrix(int k, const lbp_basis* set, int r, int8_t* P_out);
+
+/* Table 1 closed forms, in FLOPs.  which: 0 vanilla BP 4 Cx Cy L, 1 projection
+ * (Cx+Cy) L r, 2 low-rank products 4 Cx Cy r, 3 reverse projection Cx L r,
+ * 4 = 1+2+3.  Returns a negative number for a bad `which`. */
+double lbp_flops(int Cin, int Cout, long long L, int r, int which);
+
+const char* lbp_status_string(int status);
+
+/* cudaError_t (as int) of the most recent failed CUDA call made by this
+ * library on the calling thread; 0 if none. */
+int lbp_last_cuda_error(void);
+
+/* ---- device entry points ------------------------------------------------- */
+
+/* Bytes of scratch the calls below need for this layer at rank r (Algorithm 1
+ * materialises x_hat and g_y_hat; the status word lives there too).  Returns 0
+ * for an invalid layer.  lbp_project / lbp_expand need lbp_status_bytes(). */
+size_t lbp_workspace_bytes(const lbp_layer* layer, int r);
+size_t lbp_status_bytes(void);
+
+/* Eq. 6 per block:  t_hat[b,bh,bw,q,c] = (1/k) sum_{u,v} wal_iq[u] wal_jq[v]
+ *                                         t[b, bh*k+u, bw*k+v, c].
+ * t (B,H,W,C) -> t_hat (B,H/k,W/k,r,C), both of `dtype`; fp32 accumulation,
+ * one rounding to the output type.  ws: >= lbp_status_bytes(). */
+int lbp_project(const void* t, void* t_hat, int B, int H, int W, int C, int k,
+                const lbp_basis* set, int r, int dtype,
+                void* ws, size_t ws_bytes, void* stream);
+
+/* Eq. 7 per block:  t[b,bh*k+u,bw*k+v,c] = (1/k) sum_q wal_iq[u] wal_jq[v]
+ *                                          t_hat[b,bh,bw,q,c].
+ * t_hat (B,H/k,W/k,r,C) -> t (B,H,W,C), both of `dtype`. */
+int lbp_expand(const void* t_hat, void* t, int B, int H, int W, int C, int k,
+               const lbp_basis* set, int r, int dtype,
+               void* ws, size_t ws_bytes, void* stream);
+
+/* Algorithm 1:  x_hat = p(x), g_y_hat = p(g_y), g_W = g_y_hat^T x_hat (summed
+ * over batch, blocks and bases), g_x_hat = g_y_hat W, g_x = p^-1(g_x_hat).
+ * g_x and g_W are overwritten.  With bf16 data x_hat and g_y_hat are rounded to
+ * bf16, products accumulate in fp32, g_x_hat stays fp32 until g_x is rounded
+ * once.  r == k*k (any order of the complete set) runs the full-rank mode.
+ * ws: >= lbp_workspace_bytes(layer, r). */
+int lbp_backward(const void* x, const void* g_y, const void* W,
+                 void* g_x, void* g_W, const lbp_layer* layer,
+                 const lbp_basis* set, int r,
+                 void* ws, size_t ws_bytes, void* stream);
+
+/* Eq. 2, exact backpropagation: g_W = g_y^T x over all tokens, g_x = g_y W.
+ * This is what all k*k bases give (P P^T = I), computed without transforms.
+ * ws: >= lbp_workspace_bytes(layer, k*k). */
+int lbp_backward_fullrank(const void* x, const void* g_y, const void* W,
+                          void* g_x, void* g_W, const lbp_layer* layer,
+                          void* ws, size_t ws_bytes, void* stream);
+
+/* Synchronises `stream`, reads the device status word at the start of ws and
+ * clears it.  Returns LBP_OK, LBP_ERR_TIMEOUT (a bounded wait in a kernel
+ * expired; outputs of that call are undefined, the context stays usable) or
+ * LBP_ERR_CUDA. */
+int lbp_poll_status(void* ws, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LBP_H_ */

@@ -1,0 +1,97 @@
+// Internal declarations shared by the translation units of liblbp:
+// host-side plan structures, launch prototypes and error plumbing.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "lbp.h"
+
+namespace lbp {
+
+constexpr int kMaxOrder = 16;                    // largest WHT order k
+constexpr int kMaxRank = kMaxOrder * kMaxOrder;  // r <= k*k
+
+// Device status block at the start of every workspace (256 B reserved).
+//   word 0: an lbp_status (LBP_ERR_TIMEOUT) written by a kernel whose wait expired
+//   word 1: where that wait gave up (kernel id << 16 | site)
+//   word 2: kStatusMagic, written together with word 0; the block counts as
+//           "no error" unless the magic is present, so the caller's scratch
+//           needs no initialisation.
+constexpr size_t kStatusBytes = 256;
+constexpr uint32_t kStatusMagic = 0x4C425045u;
+
+// A validated basis list, prepared for the transform kernels.
+//
+// The kernels pool each k x k block down to LB x LB (LB = smallest power of two
+// above the largest selected index; Walsh rows of sequency < LB are constant on
+// runs of k/LB), run an LB x LB Hadamard butterfly in natural (Sylvester) order
+// and pick the selected coefficients.  `qmap` maps a natural-order position
+// (a, b) of that LB x LB array to the slot q of the basis list, -1 = unused.
+struct BasisPlan {
+  int32_t k;
+  int32_t r;
+  int32_t LB;
+  int16_t qmap[kMaxRank];  // [a * LB + b]
+};
+
+// Validates (k, set, r) and fills `plan`.  Returns an lbp_status.
+int make_basis_plan(int k, const lbp_basis* set, int r, BasisPlan* plan);
+
+// Natural (Sylvester) row index of the length-n Walsh row with s sign changes.
+int walsh_natural_index(int n, int s);
+// wal_s[u] for order k: +1 or -1.
+int walsh_sign(int k, int s, int u);
+
+int check_order(int k);
+
+void set_last_cuda_error(cudaError_t e);
+#define LBP_CUDA_TRY(expr)                       \
+  do {                                           \
+    cudaError_t e__ = (expr);                    \
+    if (e__ != cudaSuccess) {                    \
+      ::lbp::set_last_cuda_error(e__);           \
+      return LBP_ERR_CUDA;                       \
+    }                                            \
+  } while (0)
+
+// ---- tensor maps (TMA descriptors), encoded on the host ------------------
+// 4-D channels-last tensor (B, H, W, C): box = one k x k block x box_c
+// channels, no swizzle.
+int encode_block_tensor_map(CUtensorMap* map, const void* base, int dtype, int B, int H, int W,
+                            int C, int k, int box_c);
+// 2-D row-major bf16 matrix (rows, cols): box = box_rows x 64 columns (128 B),
+// 128-byte swizzle.
+int encode_matrix_tensor_map(CUtensorMap* map, const void* base, long long rows, long long cols,
+                             int box_rows);
+
+// ---- kernel launchers (each returns an lbp_status) ------------------------
+// Row q of block blk of a projected tensor lives at
+//   (blk / bpt) * tile_rows + (blk % bpt) * r + q ;   dense: bpt = 1, tile_rows = r.
+struct RowMap {
+  int32_t bpt;
+  int32_t tile_rows;
+};
+
+int launch_project(const void* t, void* t_hat, int dtype, int B, int H, int W, int C,
+                   const BasisPlan& plan, RowMap rows, uint32_t* status, cudaStream_t stream);
+
+// t_hat is fp32 when `in_f32`, else of `dtype`; t is of `dtype`.
+int launch_expand(const void* t_hat, bool in_f32, void* t, int dtype, int B, int H, int W, int C,
+                  const BasisPlan& plan, RowMap rows, cudaStream_t stream);
+
+// D[M, N] = sum_k A(m, k) * B(k, n), fp32 accumulation.
+//   a_mn_major == false: A is stored (M, K) row-major;  true: A is stored (K, M) row-major.
+//   B is stored (K, N) row-major.  D is (M, N) row-major of d_dtype.
+// bf16 operands run on tcgen05 tensor cores; fp32 operands on FFMA.
+// `splitk_ws` holds fp32 partial tiles when the kernel splits K.
+int launch_gemm(const void* A, bool a_mn_major, const void* Bm, void* D, int in_dtype, int d_dtype,
+                long long M, long long N, long long K, float* splitk_ws, size_t splitk_ws_bytes,
+                uint32_t* status, cudaStream_t stream);
+size_t gemm_splitk_ws_bytes(long long M, long long N, long long K, int in_dtype);
+
+int check_device_arch();
+
+}  // namespace lbp
