@@ -1,0 +1,244 @@
+"""ctypes binding of liblbp.so: argument marshalling only.
+
+Every function mirrors one entry point of include/lbp.h.  Tensors are torch
+CUDA tensors used as device-memory handles (data_ptr) -- all arithmetic runs in
+the library's kernels.  There is no CPU or eager fallback: if the shared library
+is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblbp.so")
+
+LBP_F32, LBP_BF16 = 0, 1
+SEL_L1, SEL_LINF, SEL_PREFIX = 0, 1, 2
+LBP_OK = 0
+
+
+class LbpError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = _lib().lbp_status_string(status).decode()
+        if status == 9:
+            msg += f" (cudaError {_lib().lbp_last_cuda_error()})"
+        super().__init__(f"{where}: {msg} [status {status}]")
+
+
+class Basis(C.Structure):
+    _fields_ = [("i", C.c_int32), ("j", C.c_int32)]
+
+
+class Layer(C.Structure):
+    _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("W", C.c_int32),
+                ("Cin", C.c_int32), ("Cout", C.c_int32), ("k", C.c_int32),
+                ("dtype", C.c_int32), ("gw_dtype", C.c_int32)]
+
+
+_LIB = None
+
+
+def _lib() -> C.CDLL:
+    global _LIB
+    if _LIB is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with "
+                "`python -m paper_2309_15275_b200.build` (there is no fallback path)")
+        lib = C.CDLL(LIB_PATH)
+        vp, sz, i32 = C.c_void_p, C.c_size_t, C.c_int
+        lib.lbp_select_bases.argtypes = [i32, i32, i32, C.POINTER(Basis), i32, C.POINTER(i32)]
+        lib.lbp_select_bases.restype = i32
+        lib.lbp_basis_matrix.argtypes = [i32, C.POINTER(Basis), i32, C.POINTER(C.c_int8)]
+        lib.lbp_basis_matrix.restype = i32
+        lib.lbp_flops.argtypes = [i32, i32, C.c_longlong, i32, i32]
+        lib.lbp_flops.restype = C.c_double
+        lib.lbp_status_string.argtypes = [i32]
+        lib.lbp_status_string.restype = C.c_char_p
+        lib.lbp_last_cuda_error.argtypes = []
+        lib.lbp_last_cuda_error.restype = i32
+        lib.lbp_workspace_bytes.argtypes = [C.POINTER(Layer), i32]
+        lib.lbp_workspace_bytes.restype = sz
+        lib.lbp_status_bytes.argtypes = []
+        lib.lbp_status_bytes.restype = sz
+        for name in ("lbp_project", "lbp_expand"):
+            f = getattr(lib, name)
+            f.argtypes = [vp, vp, i32, i32, i32, i32, i32, C.POINTER(Basis), i32, i32, vp, sz, vp]
+            f.restype = i32
+        lib.lbp_backward.argtypes = [vp, vp, vp, vp, vp, C.POINTER(Layer), C.POINTER(Basis), i32,
+                                     vp, sz, vp]
+        lib.lbp_backward.restype = i32
+        lib.lbp_backward_fullrank.argtypes = [vp, vp, vp, vp, vp, C.POINTER(Layer), vp, sz, vp]
+        lib.lbp_backward_fullrank.restype = i32
+        lib.lbp_poll_status.argtypes = [vp, vp]
+        lib.lbp_poll_status.restype = i32
+        _LIB = lib
+    return _LIB
+
+
+EXPORTED = ("lbp_select_bases", "lbp_basis_matrix", "lbp_flops", "lbp_status_string",
+            "lbp_last_cuda_error", "lbp_workspace_bytes", "lbp_status_bytes", "lbp_project",
+            "lbp_expand", "lbp_backward", "lbp_backward_fullrank", "lbp_poll_status")
+
+
+def _check(status: int, where: str) -> None:
+    if status != LBP_OK:
+        raise LbpError(status, where)
+
+
+def _bases(bases: Sequence[Tuple[int, int]]):
+    arr = (Basis * max(len(bases), 1))()
+    for q, (i, j) in enumerate(bases):
+        arr[q].i, arr[q].j = int(i), int(j)
+    return arr
+
+
+def _dtype_code(t: torch.dtype) -> int:
+    if t == torch.float32:
+        return LBP_F32
+    if t == torch.bfloat16:
+        return LBP_BF16
+    raise TypeError(f"unsupported dtype {t}")
+
+
+def _dev(t: torch.Tensor, name: str) -> int:
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (the library has no CPU path)")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+# ------------------------------------------------------------ host helpers ----
+def lbp_select_bases(k: int, rule: int, param: int) -> List[Tuple[int, int]]:
+    out = (Basis * 256)()
+    r = C.c_int(0)
+    _check(_lib().lbp_select_bases(k, rule, param, out, 256, C.byref(r)), "lbp_select_bases")
+    return [(out[q].i, out[q].j) for q in range(r.value)]
+
+
+def lbp_basis_matrix(k: int, bases: Sequence[Tuple[int, int]]):
+    import numpy as np
+    r = len(bases)
+    buf = (C.c_int8 * (k * k * max(r, 1)))()
+    _check(_lib().lbp_basis_matrix(k, _bases(bases), r, buf), "lbp_basis_matrix")
+    return np.frombuffer(buf, dtype=np.int8).reshape(k * k, r).copy()
+
+
+def lbp_flops(Cin: int, Cout: int, L: int, r: int, which: int) -> float:
+    return float(_lib().lbp_flops(Cin, Cout, L, r, which))
+
+
+def lbp_status_string(status: int) -> str:
+    return _lib().lbp_status_string(status).decode()
+
+
+def lbp_status_bytes() -> int:
+    return int(_lib().lbp_status_bytes())
+
+
+def _layer(B, H, W, Cin, Cout, k, dtype, gw_dtype) -> Layer:
+    return Layer(B, H, W, Cin, Cout, k, dtype, gw_dtype)
+
+
+def lbp_workspace_bytes(B, H, W, Cin, Cout, k, dtype: int, gw_dtype: int, r: int) -> int:
+    lay = _layer(B, H, W, Cin, Cout, k, dtype, gw_dtype)
+    return int(_lib().lbp_workspace_bytes(C.byref(lay), r))
+
+
+# ---------------------------------------------------------- device calls ----
+def _status_ws(device) -> torch.Tensor:
+    return torch.empty(lbp_status_bytes(), dtype=torch.uint8, device=device)
+
+
+def lbp_project(t: torch.Tensor, k: int, bases, out: torch.Tensor | None = None,
+                ws: torch.Tensor | None = None) -> torch.Tensor:
+    """t (B,H,W,C) -> t_hat (B,H/k,W/k,r,C)."""
+    B, H, W, Cc = t.shape
+    r = len(bases)
+    if out is None:
+        out = torch.empty((B, H // max(k, 1), W // max(k, 1), r, Cc), dtype=t.dtype, device=t.device)
+    if ws is None:
+        ws = _status_ws(t.device)
+    _check(_lib().lbp_project(_dev(t, "t"), _dev(out, "t_hat"), B, H, W, Cc, k, _bases(bases), r,
+                              _dtype_code(t.dtype), _dev(ws, "ws"), ws.numel(), _stream()),
+           "lbp_project")
+    return out
+
+
+def lbp_expand(t_hat: torch.Tensor, k: int, bases, out: torch.Tensor | None = None,
+               ws: torch.Tensor | None = None) -> torch.Tensor:
+    """t_hat (B,H/k,W/k,r,C) -> t (B,H,W,C)."""
+    B, Hb, Wb, r, Cc = t_hat.shape
+    if out is None:
+        out = torch.empty((B, Hb * k, Wb * k, Cc), dtype=t_hat.dtype, device=t_hat.device)
+    if ws is None:
+        ws = _status_ws(t_hat.device)
+    _check(_lib().lbp_expand(_dev(t_hat, "t_hat"), _dev(out, "t"), B, Hb * k, Wb * k, Cc, k,
+                             _bases(bases), len(bases), _dtype_code(t_hat.dtype),
+                             _dev(ws, "ws"), ws.numel(), _stream()),
+           "lbp_expand")
+    return out
+
+
+def alloc_workspace(x: torch.Tensor, g_y: torch.Tensor, k: int, r: int,
+                    gw_dtype: torch.dtype = torch.float32) -> torch.Tensor:
+    B, H, W, Cin = x.shape
+    n = lbp_workspace_bytes(B, H, W, Cin, g_y.shape[-1], k, _dtype_code(x.dtype),
+                            _dtype_code(gw_dtype), r)
+    if n == 0:
+        raise ValueError("invalid layer for lbp_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=x.device)
+
+
+def lbp_backward(x, g_y, W, k: int, bases, *, gw_dtype: torch.dtype = torch.float32,
+                 g_x=None, g_W=None, ws=None):
+    """Algorithm 1.  Returns (g_x (B,H,W,Cin), g_W (Cout,Cin))."""
+    B, H, Wd, Cin = x.shape
+    Cout = g_y.shape[-1]
+    r = len(bases)
+    if g_x is None:
+        g_x = torch.empty_like(x)
+    if g_W is None:
+        g_W = torch.empty((Cout, Cin), dtype=gw_dtype, device=x.device)
+    if ws is None:
+        ws = alloc_workspace(x, g_y, k, r, g_W.dtype)
+    lay = _layer(B, H, Wd, Cin, Cout, k, _dtype_code(x.dtype), _dtype_code(g_W.dtype))
+    _check(_lib().lbp_backward(_dev(x, "x"), _dev(g_y, "g_y"), _dev(W, "W"), _dev(g_x, "g_x"),
+                               _dev(g_W, "g_W"), C.byref(lay), _bases(bases), r,
+                               _dev(ws, "ws"), ws.numel(), _stream()),
+           "lbp_backward")
+    return g_x, g_W
+
+
+def lbp_backward_fullrank(x, g_y, W, k: int, *, gw_dtype: torch.dtype = torch.float32,
+                          g_x=None, g_W=None, ws=None):
+    """Eq. 2, exact backpropagation (the r = k*k mode)."""
+    B, H, Wd, Cin = x.shape
+    Cout = g_y.shape[-1]
+    if g_x is None:
+        g_x = torch.empty_like(x)
+    if g_W is None:
+        g_W = torch.empty((Cout, Cin), dtype=gw_dtype, device=x.device)
+    if ws is None:
+        ws = alloc_workspace(x, g_y, k, k * k, g_W.dtype)
+    lay = _layer(B, H, Wd, Cin, Cout, k, _dtype_code(x.dtype), _dtype_code(g_W.dtype))
+    _check(_lib().lbp_backward_fullrank(_dev(x, "x"), _dev(g_y, "g_y"), _dev(W, "W"),
+                                        _dev(g_x, "g_x"), _dev(g_W, "g_W"), C.byref(lay),
+                                        _dev(ws, "ws"), ws.numel(), _stream()),
+           "lbp_backward_fullrank")
+    return g_x, g_W
+
+
+def lbp_poll_status(ws: torch.Tensor) -> int:
+    """Synchronises the current stream and returns the device status (0 = ok)."""
+    return int(_lib().lbp_poll_status(_dev(ws, "ws"), _stream()))

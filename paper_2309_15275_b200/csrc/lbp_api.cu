@@ -1,0 +1,264 @@
+// C-ABI entry points that touch the device: argument validation, workspace
+// layout, TMA descriptor encoding and the launch sequence of Algorithm 1.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "lbp_internal.h"
+
+namespace lbp {
+
+// ---------------------------------------------------------------- helpers ----
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+static int elem_size(int dtype) { return dtype == LBP_BF16 ? 2 : 4; }
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_device_arch() {
+  int dev = 0, major = 0;
+  LBP_CUDA_TRY(cudaGetDevice(&dev));
+  LBP_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+  return major == 10 ? LBP_OK : LBP_ERR_ARCH;
+}
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver entry point is resolved at run time so that the library loads
+// (for its host-only functions) on machines without a CUDA driver.
+static int get_encode_fn(EncodeTiledFn* out) {
+  static EncodeTiledFn cached = nullptr;
+  if (cached == nullptr) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    LBP_CUDA_TRY(cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000,
+                                                  cudaEnableDefault, &qres));
+    if (qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+      set_last_cuda_error(cudaErrorNotSupported);
+      return LBP_ERR_CUDA;
+    }
+    cached = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  *out = cached;
+  return LBP_OK;
+}
+
+int encode_block_tensor_map(CUtensorMap* map, const void* base, int dtype, int B, int H, int W,
+                            int C, int k, int box_c) {
+  EncodeTiledFn enc;
+  if (int e = get_encode_fn(&enc)) return e;
+  const cuuint64_t es = static_cast<cuuint64_t>(elem_size(dtype));
+  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W),
+                              static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(B)};
+  const cuuint64_t strides[3] = {dims[0] * es, dims[0] * dims[1] * es,
+                                 dims[0] * dims[1] * dims[2] * es};
+  const cuuint32_t box[4] = {static_cast<cuuint32_t>(box_c), static_cast<cuuint32_t>(k),
+                             static_cast<cuuint32_t>(k), 1u};
+  const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  const CUresult r =
+      enc(map, dtype == LBP_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+          4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+          CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error(cudaErrorInvalidValue);
+    return LBP_ERR_CUDA;
+  }
+  return LBP_OK;
+}
+
+int encode_matrix_tensor_map(CUtensorMap* map, const void* base, long long rows, long long cols,
+                             int box_rows) {
+  EncodeTiledFn enc;
+  if (int e = get_encode_fn(&enc)) return e;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * 2};
+  const cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t estr[2] = {1u, 1u};
+  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+                         strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error(cudaErrorInvalidValue);
+    return LBP_ERR_CUDA;
+  }
+  return LBP_OK;
+}
+
+static int check_grid(int B, int H, int W, int C, int k, int dtype) {
+  if (int e = check_order(k)) return e;
+  if (dtype != LBP_F32 && dtype != LBP_BF16) return LBP_ERR_DTYPE;
+  if (B <= 0 || H <= 0 || W <= 0 || C <= 0) return LBP_ERR_SHAPE;
+  if (H % k != 0 || W % k != 0) return LBP_ERR_SHAPE;
+  if ((static_cast<long long>(C) * elem_size(dtype)) % 16 != 0) return LBP_ERR_ALIGN;
+  return LBP_OK;
+}
+
+static int check_layer(const lbp_layer* L) {
+  if (L == nullptr) return LBP_ERR_NULL;
+  if (int e = check_grid(L->B, L->H, L->W, L->Cin, L->k, L->dtype)) return e;
+  if (int e = check_grid(L->B, L->H, L->W, L->Cout, L->k, L->dtype)) return e;
+  if (L->gw_dtype != LBP_F32 && L->gw_dtype != LBP_BF16) return LBP_ERR_DTYPE;
+  if (L->dtype == LBP_F32 && L->gw_dtype != LBP_F32) return LBP_ERR_DTYPE;
+  return LBP_OK;
+}
+
+// Workspace layout of lbp_backward at rank r < k*k.
+struct Layout {
+  size_t x_hat, gy_hat, gx_hat, splitk, splitk_bytes, total;
+  long long rows;   // M_hat = blocks * r
+};
+
+static Layout plan_layout(const lbp_layer& L, int r) {
+  Layout w{};
+  const long long T = static_cast<long long>(L.B) * L.H * L.W;
+  const long long nb = T / (L.k * L.k);
+  const int es = elem_size(L.dtype);
+  size_t off = kStatusBytes;
+  if (r < L.k * L.k) {
+    w.rows = nb * r;
+    w.x_hat = off = align_up(off, 1024);
+    off += static_cast<size_t>(w.rows) * L.Cin * es;
+    w.gy_hat = off = align_up(off, 1024);
+    off += static_cast<size_t>(w.rows) * L.Cout * es;
+    w.gx_hat = off = align_up(off, 1024);
+    off += static_cast<size_t>(w.rows) * L.Cin * 4;
+    const size_t a = gemm_splitk_ws_bytes(L.Cout, L.Cin, w.rows, L.dtype);
+    const size_t b = gemm_splitk_ws_bytes(w.rows, L.Cin, L.Cout, L.dtype);
+    w.splitk_bytes = a > b ? a : b;
+  } else {
+    w.rows = T;
+    const size_t a = gemm_splitk_ws_bytes(L.Cout, L.Cin, T, L.dtype);
+    const size_t b = gemm_splitk_ws_bytes(T, L.Cin, L.Cout, L.dtype);
+    w.splitk_bytes = a > b ? a : b;
+  }
+  w.splitk = off = align_up(off, 1024);
+  off += w.splitk_bytes;
+  w.total = align_up(off, 256);
+  return w;
+}
+
+static int run_fullrank(const void* x, const void* g_y, const void* W, void* g_x, void* g_W,
+                        const lbp_layer& L, uint8_t* ws, cudaStream_t stream) {
+  const Layout lay = plan_layout(L, L.k * L.k);
+  const long long T = lay.rows;
+  uint32_t* status = reinterpret_cast<uint32_t*>(ws);
+  float* sk = reinterpret_cast<float*>(ws + lay.splitk);
+  // Eq. 2: g_W = g_y^T x
+  if (int e = launch_gemm(g_y, /*a_mn_major=*/true, x, g_W, L.dtype, L.gw_dtype, L.Cout, L.Cin, T,
+                          sk, lay.splitk_bytes, status, stream))
+    return e;
+  // Eq. 2: g_x = g_y W
+  return launch_gemm(g_y, /*a_mn_major=*/false, W, g_x, L.dtype, L.dtype, T, L.Cin, L.Cout, sk,
+                     lay.splitk_bytes, status, stream);
+}
+
+}  // namespace lbp
+
+using namespace lbp;
+
+extern "C" {
+
+size_t lbp_workspace_bytes(const lbp_layer* layer, int r) {
+  if (check_layer(layer) != LBP_OK) return 0;
+  if (r < 1 || r > layer->k * layer->k) return 0;
+  return plan_layout(*layer, r).total;
+}
+
+int lbp_project(const void* t, void* t_hat, int B, int H, int W, int C, int k,
+                const lbp_basis* set, int r, int dtype, void* ws, size_t ws_bytes, void* stream) {
+  if (t == nullptr || t_hat == nullptr) return LBP_ERR_NULL;
+  if (int e = check_grid(B, H, W, C, k, dtype)) return e;
+  BasisPlan plan;
+  if (int e = make_basis_plan(k, set, r, &plan)) return e;
+  if (!aligned16(t) || !aligned16(t_hat) || !aligned16(ws)) return LBP_ERR_ALIGN;
+  if (ws == nullptr || ws_bytes < kStatusBytes) return LBP_ERR_WORKSPACE;
+  if (int e = check_device_arch()) return e;
+  return launch_project(t, t_hat, dtype, B, H, W, C, plan, RowMap{1, r},
+                        static_cast<uint32_t*>(ws), static_cast<cudaStream_t>(stream));
+}
+
+int lbp_expand(const void* t_hat, void* t, int B, int H, int W, int C, int k,
+               const lbp_basis* set, int r, int dtype, void* ws, size_t ws_bytes, void* stream) {
+  if (t == nullptr || t_hat == nullptr) return LBP_ERR_NULL;
+  if (int e = check_grid(B, H, W, C, k, dtype)) return e;
+  BasisPlan plan;
+  if (int e = make_basis_plan(k, set, r, &plan)) return e;
+  if (!aligned16(t) || !aligned16(t_hat) || !aligned16(ws)) return LBP_ERR_ALIGN;
+  if (ws == nullptr || ws_bytes < kStatusBytes) return LBP_ERR_WORKSPACE;
+  if (int e = check_device_arch()) return e;
+  return launch_expand(t_hat, /*in_f32=*/dtype == LBP_F32, t, dtype, B, H, W, C, plan,
+                       RowMap{1, r}, static_cast<cudaStream_t>(stream));
+}
+
+int lbp_backward(const void* x, const void* g_y, const void* W, void* g_x, void* g_W,
+                 const lbp_layer* layer, const lbp_basis* set, int r, void* ws, size_t ws_bytes,
+                 void* stream) {
+  if (x == nullptr || g_y == nullptr || W == nullptr || g_x == nullptr || g_W == nullptr)
+    return LBP_ERR_NULL;
+  if (int e = check_layer(layer)) return e;
+  const lbp_layer& L = *layer;
+  BasisPlan plan;
+  if (int e = make_basis_plan(L.k, set, r, &plan)) return e;
+  if (!aligned16(x) || !aligned16(g_y) || !aligned16(W) || !aligned16(g_x) || !aligned16(g_W) ||
+      !aligned16(ws))
+    return LBP_ERR_ALIGN;
+  const Layout lay = plan_layout(L, r);
+  if (ws == nullptr || ws_bytes < lay.total) return LBP_ERR_WORKSPACE;
+  if (int e = check_device_arch()) return e;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* wsb = static_cast<uint8_t*>(ws);
+  if (r == L.k * L.k) return run_fullrank(x, g_y, W, g_x, g_W, L, wsb, st);
+
+  uint32_t* status = reinterpret_cast<uint32_t*>(wsb);
+  void* x_hat = wsb + lay.x_hat;
+  void* gy_hat = wsb + lay.gy_hat;
+  float* gx_hat = reinterpret_cast<float*>(wsb + lay.gx_hat);
+  float* sk = reinterpret_cast<float*>(wsb + lay.splitk);
+  const RowMap dense{1, r};
+
+  // Algorithm 1, steps 1-2: x_hat = p(x), g_y_hat = p(g_y)
+  if (int e = launch_project(x, x_hat, L.dtype, L.B, L.H, L.W, L.Cin, plan, dense, status, st))
+    return e;
+  if (int e = launch_project(g_y, gy_hat, L.dtype, L.B, L.H, L.W, L.Cout, plan, dense, status, st))
+    return e;
+  // step 3: g_W = g_y_hat^T x_hat
+  if (int e = launch_gemm(gy_hat, /*a_mn_major=*/true, x_hat, g_W, L.dtype, L.gw_dtype, L.Cout,
+                          L.Cin, lay.rows, sk, lay.splitk_bytes, status, st))
+    return e;
+  // step 4: g_x_hat = g_y_hat W   (kept in fp32)
+  if (int e = launch_gemm(gy_hat, /*a_mn_major=*/false, W, gx_hat, L.dtype, LBP_F32, lay.rows,
+                          L.Cin, L.Cout, sk, lay.splitk_bytes, status, st))
+    return e;
+  // step 5: g_x = p^-1(g_x_hat)
+  return launch_expand(gx_hat, /*in_f32=*/true, g_x, L.dtype, L.B, L.H, L.W, L.Cin, plan, dense, st);
+}
+
+int lbp_backward_fullrank(const void* x, const void* g_y, const void* W, void* g_x, void* g_W,
+                          const lbp_layer* layer, void* ws, size_t ws_bytes, void* stream) {
+  if (x == nullptr || g_y == nullptr || W == nullptr || g_x == nullptr || g_W == nullptr)
+    return LBP_ERR_NULL;
+  if (int e = check_layer(layer)) return e;
+  if (!aligned16(x) || !aligned16(g_y) || !aligned16(W) || !aligned16(g_x) || !aligned16(g_W) ||
+      !aligned16(ws))
+    return LBP_ERR_ALIGN;
+  const Layout lay = plan_layout(*layer, layer->k * layer->k);
+  if (ws == nullptr || ws_bytes < lay.total) return LBP_ERR_WORKSPACE;
+  if (int e = check_device_arch()) return e;
+  return run_fullrank(x, g_y, W, g_x, g_W, *layer, static_cast<uint8_t*>(ws),
+                      static_cast<cudaStream_t>(stream));
+}
+
+int lbp_poll_status(void* ws, void* stream) {
+  if (ws == nullptr) return LBP_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  LBP_CUDA_TRY(cudaStreamSynchronize(st));
+  uint32_t words[4] = {0, 0, 0, 0};
+  LBP_CUDA_TRY(cudaMemcpy(words, ws, sizeof(words), cudaMemcpyDeviceToHost));
+  if (words[2] != kStatusMagic) return LBP_OK;
+  LBP_CUDA_TRY(cudaMemset(ws, 0, sizeof(words)));
+  return words[0] == 0 ? LBP_OK : static_cast<int>(words[0]);
+}
+
+}  // extern "C"

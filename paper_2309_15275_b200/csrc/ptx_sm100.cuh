@@ -53,12 +53,13 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint64_t* bar, uint32_t parity
   return done;
 }
 
-// Report an expired wait: first failure wins, later ones leave it alone.
+// Report an expired wait: the first reporter wins.  The status block needs no
+// initialisation: it only counts as an error once the magic word is present.
 __device__ __forceinline__ void report_timeout(uint32_t* status, uint32_t site) {
-  if (status != nullptr && atomicCAS(status, 0u, static_cast<uint32_t>(LBP_ERR_TIMEOUT)) == 0u) {
+  if (status != nullptr && atomicExch(status + 2, kStatusMagic) != kStatusMagic) {
+    status[0] = static_cast<uint32_t>(LBP_ERR_TIMEOUT);
     status[1] = site;
     __threadfence();
-    status[2] = kStatusMagic;
   }
 }
 

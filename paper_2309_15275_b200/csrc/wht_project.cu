@@ -1,0 +1,291 @@
+// Projection kernel (Eq. 6):  t_hat[blk, q, c] = (1/k) sum_{u,v} wal_iq[u] wal_jq[v] t[blk,u,v,c].
+//
+// HBM-bound streaming pass.  One warp owns a ring of shared-memory stages; lane
+// 0 issues one 4-D TMA box per (block, channel chunk) -- k x k tokens by 128
+// bytes of channels -- and the warp consumes it with conflict-free 32-bit
+// shared loads (a lane owns one word of the channel axis).  The transform is
+// additions only: pool to LB x LB, then a natural-order Hadamard butterfly.
+#include <cuda_bf16.h>
+
+#include "lbp_internal.h"
+#include "ptx_sm100.cuh"
+#include "wht_device.cuh"
+
+namespace lbp {
+
+struct ProjParams {
+  int32_t nb, Hb, Wb, C, r, n_chunks;
+  int32_t bpt, tile_rows;
+  long long n_items;   // nb * n_chunks
+  uint32_t* status;
+  float scale;         // 1/k
+};
+
+template <int K, bool BF16>
+struct ProjCfg {
+  static constexpr int kTileBytesMax = K * K * 128;
+  static constexpr int kWarps = (K == 16) ? 6 : 12;
+  static constexpr int kStages = (K == 4) ? 4 : (K == 8 ? 2 : 1);
+  static constexpr int kSmemBytes = kWarps * kStages * kTileBytesMax + kWarps * kStages * 8 + 128;
+};
+
+template <typename T, bool BF16, int NCH>
+__device__ __forceinline__ void store_coeff(T* __restrict__ out, long long row, int C, int c0,
+                                            int pass, const float (&v)[NCH], float scale) {
+  if constexpr (!BF16) {
+    out[row * C + c0] = v[0] * scale;
+  } else if constexpr (NCH == 2) {
+    *reinterpret_cast<uint32_t*>(out + row * C + c0) = pack_bf16x2(v[0] * scale, v[1] * scale);
+  } else {
+    out[row * C + c0 + pass] = __float2bfloat16_rn(v[0] * scale);
+  }
+}
+
+template <typename T, int K, int LB>
+__global__ void __launch_bounds__(ProjCfg<K, sizeof(T) == 2>::kWarps * 32, 1)
+    wht_project_kernel(const __grid_constant__ CUtensorMap tmap, T* __restrict__ out,
+                       const __grid_constant__ ProjParams p,
+                       const __grid_constant__ DevicePlan plan) {
+  constexpr bool BF16 = sizeof(T) == 2;
+  using Cfg = ProjCfg<K, BF16>;
+  constexpr int NW = Cfg::kWarps, S = Cfg::kStages;
+  constexpr int CH_PER_WORD = BF16 ? 2 : 1;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + NW * S * Cfg::kTileBytesMax);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  uint64_t* my_bars = bars + warp * S;
+  uint8_t* my_tiles = tiles + warp * S * Cfg::kTileBytesMax;
+
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < S; ++s) ptx::mbar_init(&my_bars[s], 1);
+    ptx::mbar_fence_init();
+  }
+  if (threadIdx.x == 0) ptx::prefetch_tensormap(&tmap);
+  __syncthreads();
+
+  const long long first = static_cast<long long>(blockIdx.x) * NW + warp;
+  const long long stride = static_cast<long long>(gridDim.x) * NW;
+  const long long n_my = first < p.n_items ? (p.n_items - first + stride - 1) / stride : 0;
+  constexpr int ch_per_tile = 32 * CH_PER_WORD;   // a token is 128 B = 32 words wide in a tile
+  constexpr int tw = 32;
+
+  auto issue = [&](long long idx, int s) {
+    const long long item = first + idx * stride;
+    const int chunk = static_cast<int>(item % p.n_chunks);
+    const int blk = static_cast<int>(item / p.n_chunks);
+    const int bw = blk % p.Wb, bh = (blk / p.Wb) % p.Hb, b = blk / (p.Wb * p.Hb);
+    ptx::mbar_expect_tx(&my_bars[s], static_cast<uint32_t>(Cfg::kTileBytesMax));
+    ptx::tma_load_4d(my_tiles + s * Cfg::kTileBytesMax, &tmap, &my_bars[s], chunk * ch_per_tile,
+                     bw * K, bh * K, b);
+  };
+
+  if (lane == 0) {
+    for (int i = 0; i < S && i < n_my; ++i) issue(i, i);
+  }
+
+  for (long long idx = 0; idx < n_my; ++idx) {
+    const int s = static_cast<int>(idx % S);
+    const uint32_t parity = static_cast<uint32_t>((idx / S) & 1);
+    const bool ok = ptx::mbar_wait(&my_bars[s], parity, p.status, (1u << 16) | 1u);
+    if (!__all_sync(0xffffffffu, ok)) break;
+
+    const long long item = first + idx * stride;
+    const int chunk = static_cast<int>(item % p.n_chunks);
+    const int blk = static_cast<int>(item / p.n_chunks);
+    const uint32_t* tile = reinterpret_cast<const uint32_t*>(my_tiles + s * Cfg::kTileBytesMax);
+    const int c0 = chunk * ch_per_tile + lane * CH_PER_WORD;
+    const bool active = c0 < p.C;   // channels past C are zero-filled by TMA and skipped
+    const long long row0 =
+        static_cast<long long>(blk / p.bpt) * p.tile_rows + static_cast<long long>(blk % p.bpt) * p.r;
+
+    if (active) {
+      if constexpr (LB < 16) {
+        constexpr int RUN = K / LB;
+        constexpr int NCH = (BF16 && LB <= 4) ? 2 : 1;
+        constexpr int NPASS = (BF16 && NCH == 1) ? 2 : 1;
+#pragma unroll 1
+        for (int pass = 0; pass < NPASS; ++pass) {
+          float acc[LB][LB][NCH];
+#pragma unroll
+          for (int a = 0; a < LB; ++a)
+#pragma unroll
+            for (int b = 0; b < LB; ++b)
+#pragma unroll
+              for (int c = 0; c < NCH; ++c) acc[a][b][c] = 0.f;
+#pragma unroll
+          for (int u = 0; u < K; ++u) {
+#pragma unroll
+            for (int v = 0; v < K; ++v) {
+              float f[NCH];
+              unpack_word<BF16, NCH>(tile[(u * K + v) * tw + lane], pass, f);
+#pragma unroll
+              for (int c = 0; c < NCH; ++c) acc[u / RUN][v / RUN][c] += f[c];
+            }
+            // keep the 256 loads of an order-16 block from being hoisted together
+            if constexpr (K == 16) asm volatile("" ::: "memory");
+          }
+          hadamard_rows<LB, NCH>(acc);
+          hadamard_cols<LB, NCH>(acc);
+#pragma unroll
+          for (int a = 0; a < LB; ++a) {
+#pragma unroll
+            for (int b = 0; b < LB; ++b) {
+              const int q = plan.qmap[a * LB + b];
+              if (q >= 0) store_coeff<T, BF16, NCH>(out, row0 + q, p.C, c0, pass, acc[a][b], p.scale);
+            }
+          }
+        }
+      } else {
+        // LB == 16 (K == 16): the 16 x 16 coefficient array does not fit in
+        // registers.  Pass n_lo produces the natural-order columns
+        // b = 4 * n_hi + n_lo: a sign-combination over the low two bits of v,
+        // then a 4-point butterfly over the high two bits, then a 16-point
+        // butterfly along u.
+        constexpr int NPASS = BF16 ? 2 : 1;
+#pragma unroll 1
+        for (int pass = 0; pass < NPASS; ++pass) {
+#pragma unroll 1
+          for (int n_lo = 0; n_lo < 4; ++n_lo) {
+            const float s1 = (n_lo & 1) ? -1.f : 1.f;   // sign of v_lo = 1
+            const float s2 = (n_lo & 2) ? -1.f : 1.f;   // sign of v_lo = 2
+            const float s3 = s1 * s2;                   // sign of v_lo = 3
+            float R[4][16];                             // [n_hi][u]
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+              float y[4];
+#pragma unroll
+              for (int vh = 0; vh < 4; ++vh) {
+                float f0[1], f1[1], f2[1], f3[1];
+                unpack_word<BF16, 1>(tile[(u * 16 + vh * 4 + 0) * tw + lane], pass, f0);
+                unpack_word<BF16, 1>(tile[(u * 16 + vh * 4 + 1) * tw + lane], pass, f1);
+                unpack_word<BF16, 1>(tile[(u * 16 + vh * 4 + 2) * tw + lane], pass, f2);
+                unpack_word<BF16, 1>(tile[(u * 16 + vh * 4 + 3) * tw + lane], pass, f3);
+                y[vh] = (f0[0] + s1 * f1[0]) + (s2 * f2[0] + s3 * f3[0]);
+              }
+              hadamard_vec<4>(y);
+#pragma unroll
+              for (int nh = 0; nh < 4; ++nh) R[nh][u] = y[nh];
+              asm volatile("" ::: "memory");
+            }
+#pragma unroll
+            for (int nh = 0; nh < 4; ++nh) {
+              hadamard_vec<16>(R[nh]);
+#pragma unroll
+              for (int a = 0; a < 16; ++a) {
+                const int q = plan.qmap[a * 16 + nh * 4 + n_lo];
+                if (q >= 0) {
+                  const float v1[1] = {R[nh][a]};
+                  store_coeff<T, BF16, 1>(out, row0 + q, p.C, c0, pass, v1, p.scale);
+                }
+              }
+            }
+          }
+        }
+      }
+      // rows of a padded row tile that no block owns are kept at zero
+      if (p.bpt > 1 && ((blk % p.bpt) == p.bpt - 1 || blk == p.nb - 1)) {
+        const long long tile_base = static_cast<long long>(blk / p.bpt) * p.tile_rows;
+        for (long long row = row0 + p.r; row < tile_base + p.tile_rows; ++row) {
+          if constexpr (BF16) {
+            *reinterpret_cast<uint32_t*>(out + row * p.C + c0) = 0u;
+          } else {
+            out[row * p.C + c0] = 0.f;
+          }
+        }
+      }
+    }
+
+    __syncwarp();
+    if (lane == 0 && idx + S < n_my) {
+      ptx::fence_proxy_async_smem();
+      issue(idx + S, s);
+    }
+  }
+}
+
+template <typename T, int K, int LB>
+static int launch_one(const CUtensorMap& tmap, T* out, const ProjParams& p, const DevicePlan& plan,
+                      int sms, cudaStream_t stream) {
+  using Cfg = ProjCfg<K, sizeof(T) == 2>;
+  auto kern = wht_project_kernel<T, K, LB>;
+  static bool configured = false;
+  if (!configured) {
+    LBP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      Cfg::kSmemBytes));
+    configured = true;
+  }
+  long long want = (p.n_items + Cfg::kWarps - 1) / Cfg::kWarps;
+  const int grid = static_cast<int>(want < sms ? want : sms);
+  kern<<<grid, Cfg::kWarps * 32, Cfg::kSmemBytes, stream>>>(tmap, out, p, plan);
+  LBP_CUDA_TRY(cudaGetLastError());
+  return LBP_OK;
+}
+
+template <typename T, int K>
+static int launch_k(int LB, const CUtensorMap& tmap, T* out, const ProjParams& p,
+                    const DevicePlan& plan, int sms, cudaStream_t stream) {
+  switch (LB) {
+    case 1: return launch_one<T, K, 1>(tmap, out, p, plan, sms, stream);
+    case 2: return launch_one<T, K, 2>(tmap, out, p, plan, sms, stream);
+    case 4: return launch_one<T, K, 4>(tmap, out, p, plan, sms, stream);
+    case 8:
+      if constexpr (K >= 8) return launch_one<T, K, 8>(tmap, out, p, plan, sms, stream);
+      break;
+    case 16:
+      if constexpr (K >= 16) return launch_one<T, K, 16>(tmap, out, p, plan, sms, stream);
+      break;
+  }
+  return LBP_ERR_BASIS;
+}
+
+template <typename T>
+static int launch_t(const CUtensorMap& tmap, T* out, const ProjParams& p, const BasisPlan& bp,
+                    const DevicePlan& plan, int sms, cudaStream_t stream) {
+  switch (bp.k) {
+    case 4: return launch_k<T, 4>(bp.LB, tmap, out, p, plan, sms, stream);
+    case 8: return launch_k<T, 8>(bp.LB, tmap, out, p, plan, sms, stream);
+    case 16: return launch_k<T, 16>(bp.LB, tmap, out, p, plan, sms, stream);
+  }
+  return LBP_ERR_BLOCK;
+}
+
+int launch_project(const void* t, void* t_hat, int dtype, int B, int H, int W, int C,
+                   const BasisPlan& bp, RowMap rows, uint32_t* status, cudaStream_t stream) {
+  const int K = bp.k;
+  const int es = dtype == LBP_BF16 ? 2 : 4;
+  const int box_c = 128 / es;   // a box wider than C is legal: the excess is zero-filled
+
+  CUtensorMap tmap;
+  if (int e = encode_block_tensor_map(&tmap, t, dtype, B, H, W, C, K, box_c)) return e;
+
+  ProjParams p;
+  p.Hb = H / K;
+  p.Wb = W / K;
+  p.nb = B * p.Hb * p.Wb;
+  p.C = C;
+  p.r = bp.r;
+  p.n_chunks = (C + box_c - 1) / box_c;
+  p.bpt = rows.bpt;
+  p.tile_rows = rows.tile_rows;
+  p.n_items = static_cast<long long>(p.nb) * p.n_chunks;
+  p.status = status;
+  p.scale = 1.0f / static_cast<float>(K);
+
+  DevicePlan plan;
+  for (int n = 0; n < 256; ++n) plan.qmap[n] = bp.qmap[n];
+
+  int dev = 0, sms = 0;
+  LBP_CUDA_TRY(cudaGetDevice(&dev));
+  LBP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+
+  if (dtype == LBP_BF16)
+    return launch_t<__nv_bfloat16>(tmap, static_cast<__nv_bfloat16*>(t_hat), p, bp, plan, sms, stream);
+  return launch_t<float>(tmap, static_cast<float*>(t_hat), p, bp, plan, sms, stream);
+}
+
+}  // namespace lbp

@@ -1,0 +1,90 @@
+"""CPU-side checks of the C ABI: the library loads, exports every declared
+symbol, and its host-only functions agree with the oracle bit for bit."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2309_15275_b200 as lbp
+from oracle import lbp_oracle as O
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2309_15275_b200.build import build_library
+    build_library()
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "lbp.h")).read()
+    declared = set(re.findall(r"^(?:int|size_t|double|const char\*)\s+(lbp_[a-z_]+)\s*\(", header, re.M))
+    assert declared == set(lbp.EXPORTED)
+    lib = ctypes.CDLL(lbp.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+@pytest.mark.parametrize("k", (4, 8, 16))
+def test_select_bases_bit_exact_vs_oracle(k):
+    for m in range(1, 2 * k):
+        assert lbp.lbp_select_bases(k, lbp.SEL_L1, m) == O.select_bases(k, O.RULE_L1, m)
+    for m in range(1, k + 1):
+        assert lbp.lbp_select_bases(k, lbp.SEL_LINF, m) == O.select_bases(k, O.RULE_LINF, m)
+    for r in range(1, k * k + 1):
+        assert lbp.lbp_select_bases(k, lbp.SEL_PREFIX, r) == O.select_bases(k, O.RULE_PREFIX, r)
+
+
+@pytest.mark.parametrize("k", (4, 8, 16))
+def test_basis_matrix_bit_exact_vs_oracle(k):
+    rng = np.random.default_rng(k)
+    for r in (1, 3, k, k * k):
+        pairs = [(int(p) // k, int(p) % k) for p in rng.permutation(k * k)[:r]]
+        assert np.array_equal(lbp.lbp_basis_matrix(k, pairs), O.basis_matrix(k, pairs))
+
+
+def test_flops_match_table1():
+    f = O.flops(3072, 768, 49, 8)
+    assert lbp.lbp_flops(3072, 768, 49, 8, 0) == f["vanilla"]
+    assert lbp.lbp_flops(3072, 768, 49, 8, 1) == f["projection"]
+    assert lbp.lbp_flops(3072, 768, 49, 8, 2) == f["lowrank_mm"]
+    assert lbp.lbp_flops(3072, 768, 49, 8, 3) == f["reverse_projection"]
+    assert lbp.lbp_flops(3072, 768, 49, 8, 4) == f["projection"] + f["lowrank_mm"] + f["reverse_projection"]
+    assert lbp.lbp_flops(1, 1, 1, 1, 9) < 0
+
+
+def test_argument_errors():
+    with pytest.raises(lbp.LbpError) as e:
+        lbp.lbp_select_bases(5, lbp.SEL_L1, 2)
+    assert e.value.status == 3
+    with pytest.raises(lbp.LbpError) as e:
+        lbp.lbp_select_bases(8, lbp.SEL_PREFIX, 65)
+    assert e.value.status == 4
+    with pytest.raises(lbp.LbpError) as e:
+        lbp.lbp_basis_matrix(8, [(0, 0), (0, 0)])
+    assert e.value.status == 4
+    with pytest.raises(lbp.LbpError) as e:
+        lbp.lbp_basis_matrix(8, [(0, 8)])
+    assert e.value.status == 4
+    assert "basis" in lbp.lbp_status_string(4)
+
+
+def test_workspace_bytes():
+    n8 = lbp.lbp_workspace_bytes(128, 16, 16, 768, 3072, 8, lbp.LBP_BF16, lbp.LBP_F32, 8)
+    n16 = lbp.lbp_workspace_bytes(128, 16, 16, 768, 3072, 8, lbp.LBP_BF16, lbp.LBP_F32, 16)
+    rows = 512 * 8
+    assert n8 >= rows * (768 + 3072) * 2 + rows * 768 * 4
+    assert n16 > n8
+    assert lbp.lbp_workspace_bytes(128, 16, 12, 768, 3072, 8, lbp.LBP_BF16, lbp.LBP_F32, 8) == 0   # W % k
+    assert lbp.lbp_workspace_bytes(128, 16, 16, 768, 3072, 8, lbp.LBP_F32, lbp.LBP_BF16, 8) == 0   # dtype combo
+    assert lbp.lbp_workspace_bytes(128, 16, 16, 768, 3072, 8, lbp.LBP_BF16, lbp.LBP_F32, 65) == 0
+
+
+def test_device_calls_fail_loudly_without_cuda_tensors():
+    import torch
+    t = torch.zeros((1, 8, 8, 8), dtype=torch.float32)
+    with pytest.raises(ValueError):
+        lbp.lbp_project(t, 8, [(0, 0)], out=torch.zeros((1, 1, 1, 1, 8)), ws=torch.zeros(256, dtype=torch.uint8))
