@@ -1,0 +1,241 @@
+"""Parity of the CUDA path (through the C ABI) against the fp64 oracle.
+
+Every comparison is on the same seeded inputs, already rounded to the run
+dtype.  Bars: relative Frobenius error <= 1e-5 for fp32 data, <= 2e-2 for bf16
+data with fp32 accumulation; basis lists bit-exact (checked on the CPU suite).
+"""
+import functools
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2309_15275_b200 as lbp
+import synth
+from oracle import lbp_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+TOL = {torch.float32: 1e-5, torch.bfloat16: 2e-2}
+
+
+@pytest.fixture(scope="module")
+def dev():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    return torch.device("cuda:0")
+
+
+def f64(t):
+    return t.detach().cpu().to(torch.float64).numpy()
+
+
+def rel(got, want):
+    return O.rel_fro(f64(got), want)
+
+
+def ok_status(ws):
+    assert lbp.lbp_poll_status(ws) == 0
+
+
+@functools.lru_cache(maxsize=2)
+def _inputs(config, idx, batch):
+    return synth.make_layer_inputs(synth.config_cases(config)[idx], batch=batch)
+
+
+# ------------------------------------------------ projection / expansion ----
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("k,ranks", [(4, (1, 2, 3, 5, 16)), (8, (1, 2, 4, 6, 8, 10, 16, 21, 36, 64)),
+                                     (16, (1, 3, 8, 10, 36, 100, 256))])
+def test_project_expand_prefix_sets(dev, dtype, k, ranks):
+    # several blocks per image, ragged channel tail (C = 200 is not a multiple of a 128-byte chunk)
+    B, Hb, Wb, C = 3, 2, 3, 200
+    t = synth.make_tensor((B, Hb * k, Wb * k, C), ("normal", 1.0), "f32", case_key=700 + k).to(dtype)
+    ws = torch.zeros(lbp.lbp_status_bytes(), dtype=torch.uint8, device=dev)
+    for r in ranks:
+        bases = O.select_bases(k, O.RULE_PREFIX, r)
+        got = lbp.lbp_project(t.to(dev), k, bases, ws=ws)
+        ok_status(ws)
+        want = O.project(f64(t), k, bases)
+        assert got.shape == want.shape
+        assert rel(got, want) <= TOL[dtype], (k, r)
+        th = torch.from_numpy(want).to(dtype)
+        back = lbp.lbp_expand(th.to(dev), k, bases, ws=ws)
+        ok_status(ws)
+        assert rel(back, O.expand(f64(th), k, bases)) <= TOL[dtype], (k, r)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_project_arbitrary_sets_and_order(dev, dtype):
+    k = 8
+    t = synth.make_tensor((2, 16, 24, 72), ("normal", 1.0), "f32", case_key=710).to(dtype)
+    for bases in ([(7, 0), (0, 7), (3, 3), (1, 6), (0, 0)], [(0, 1)], [(5, 5), (2, 0)],
+                  list(reversed(O.select_bases(k, O.RULE_L1, 3))), O.select_bases(k, O.RULE_LINF, 3)):
+        got = lbp.lbp_project(t.to(dev), k, bases)
+        want = O.project(f64(t), k, bases)
+        assert rel(got, want) <= TOL[dtype], bases
+        th = torch.from_numpy(want).to(dtype)
+        back = lbp.lbp_expand(th.to(dev), k, bases)
+        assert rel(back, O.expand(f64(th), k, bases)) <= TOL[dtype], bases
+
+
+def test_project_single_block_and_narrow_channels(dev):
+    # H = W = k (one transform over the whole map), C narrower than one chunk
+    for dtype, C in ((torch.bfloat16, 8), (torch.float32, 4), (torch.bfloat16, 48)):
+        t = synth.make_tensor((1, 8, 8, C), ("normal", 1.0), "f32", case_key=720 + C).to(dtype)
+        bases = O.select_bases(8, O.RULE_L1, 4)
+        got = lbp.lbp_project(t.to(dev), 8, bases)
+        assert rel(got, O.project(f64(t), 8, bases)) <= TOL[dtype]
+
+
+def test_project_full_rank_is_lossless_fp32(dev):
+    k = 8
+    t = synth.make_tensor((2, 16, 16, 64), ("normal", 1.0), "f32", case_key=730)
+    bases = O.select_bases(k, O.RULE_PREFIX, 64)
+    th = lbp.lbp_project(t.to(dev), k, bases)
+    back = lbp.lbp_expand(th, k, bases)
+    assert rel(back, f64(t)) <= 1e-6
+
+
+def test_argument_errors_leave_outputs_untouched(dev):
+    t = torch.zeros((1, 8, 8, 8), dtype=torch.float32, device=dev)
+    out = torch.full((1, 1, 1, 1, 8), 7.0, dtype=torch.float32, device=dev)
+    ws = torch.zeros(256, dtype=torch.uint8, device=dev)
+    for k, bases, status in ((8, [(0, 0), (0, 0)], 4), (8, [(8, 0)], 4), (5, [(0, 0)], 3)):
+        with pytest.raises(lbp.LbpError) as e:
+            lbp.lbp_project(t, k, bases, out=out, ws=ws)
+        assert e.value.status == status
+    with pytest.raises(lbp.LbpError) as e:      # W % k != 0
+        lbp.lbp_project(torch.zeros((1, 8, 12, 8), device=dev), 8, [(0, 0)], out=out, ws=ws)
+    assert e.value.status == 2
+    with pytest.raises(lbp.LbpError) as e:      # C * 4 bytes not a multiple of 16
+        lbp.lbp_project(torch.zeros((1, 8, 8, 6), device=dev), 8, [(0, 0)], out=out, ws=ws)
+    assert e.value.status == 6
+    with pytest.raises(lbp.LbpError) as e:      # workspace too small
+        lbp.lbp_project(t, 8, [(0, 0)], out=out, ws=ws[:16])
+    assert e.value.status == 7
+    torch.cuda.synchronize()
+    assert torch.all(out == 7.0)
+
+
+# ------------------------------------------------------------ backward ----
+def _run_backward(dev, case, r, batch=None, fullrank_entry=False, bases=None, idx=None):
+    x, gy, w = _inputs(case.config, case.case_id if idx is None else idx, batch)
+    k = case.k
+    if bases is None:
+        bases = O.select_bases(k, O.RULE_PREFIX, r)
+    xd, gd, wd = x.to(dev), gy.to(dev), w.to(dev)
+    ws = lbp.alloc_workspace(xd, gd, k, k * k if fullrank_entry else len(bases))
+    if fullrank_entry:
+        gx, gw = lbp.lbp_backward_fullrank(xd, gd, wd, k, ws=ws)
+    else:
+        gx, gw = lbp.lbp_backward(xd, gd, wd, k, bases, ws=ws)
+    ok_status(ws)
+    return (x, gy, w), bases, gx, gw
+
+
+def _check_lowrank(dev, case, r, batch=None, bases=None):
+    (x, gy, w), bases, gx, gw = _run_backward(dev, case, r, batch, bases=bases)
+    ox, ow = O.backward_lowrank(f64(x), f64(gy), f64(w), case.k, bases)
+    tol = TOL[x.dtype]
+    assert rel(gx, ox) <= tol, (case.name, r, "g_x")
+    assert rel(gw, ow) <= tol, (case.name, r, "g_W")
+
+
+def test_config1_fp32(dev):
+    case = synth.config_cases(1)[0]
+    _check_lowrank(dev, case, 4)
+    # full rank, through the generic entry and through the full-rank entry, equals exact BP
+    x, gy, w = _inputs(1, 0, None)
+    ex, ew = O.backward_exact(f64(x), f64(gy), f64(w))
+    for entry in (False, True):
+        _, _, gx, gw = _run_backward(dev, case, 64, fullrank_entry=entry)
+        assert rel(gx, ex) <= 1e-5 and rel(gw, ew) <= 1e-5
+
+
+@pytest.mark.parametrize("k,r", [(4, 3), (4, 9), (8, 10), (8, 40), (16, 6), (16, 130)])
+def test_fp32_other_orders_and_ranks(dev, k, r):
+    case = synth.LayerCase(1, f"fp32_k{k}", 2, 2 * k, 3 * k, 40, 72, k, (r,), "f32",
+                           ("normal", 1.0), ("normal", 1.0), 3)
+    x, gy, w = synth.make_layer_inputs(case)
+    bases = O.select_bases(k, O.RULE_PREFIX, r)
+    gx, gw = lbp.lbp_backward(x.to(dev), gy.to(dev), w.to(dev), k, bases)
+    ox, ow = O.backward_lowrank(f64(x), f64(gy), f64(w), k, bases)
+    assert rel(gx, ox) <= 1e-5 and rel(gw, ow) <= 1e-5
+
+
+@pytest.mark.parametrize("idx", [0, 1])
+def test_config2_efficientformer_full_size(dev, idx):
+    _check_lowrank(dev, synth.config_cases(2)[idx], 8)
+
+
+@pytest.mark.parametrize("idx,ranks", [(0, (8,)), (1, (2, 4, 8, 16)), (2, (8, 16)), (3, (2, 8))])
+def test_config3_vitb_full_size(dev, idx, ranks):
+    case = synth.config_cases(3)[idx]
+    for r in ranks:
+        _check_lowrank(dev, case, r)
+
+
+@pytest.mark.parametrize("idx", [0, 1])
+def test_config4_vitl_full_size(dev, idx):
+    _check_lowrank(dev, synth.config_cases(4)[idx], 6)
+
+
+def test_bf16_ragged_rows_and_small_batches(dev):
+    # M_hat not a multiple of the 128-row MMA tile, K not a multiple of 64
+    case = synth.config_cases(3)[1]
+    for batch, r in ((1, 3), (3, 10), (5, 21)):
+        _check_lowrank(dev, case, r, batch=batch)
+    odd = synth.LayerCase(3, "odd", 3, 16, 24, 200, 328, 8, (5,), "bf16",
+                          ("normal", 1.0), ("normal", 0.01), 9)
+    x, gy, w = synth.make_layer_inputs(odd)
+    bases = O.select_bases(8, O.RULE_L1, 3)
+    gx, gw = lbp.lbp_backward(x.to(dev), gy.to(dev), w.to(dev), 8, bases)
+    ox, ow = O.backward_lowrank(f64(x), f64(gy), f64(w), 8, bases)
+    assert rel(gx, ox) <= 2e-2 and rel(gw, ow) <= 2e-2
+
+
+def test_bf16_gw_in_bf16(dev):
+    case = synth.config_cases(3)[1]
+    x, gy, w = _inputs(3, 1, 8)
+    bases = O.select_bases(8, O.RULE_PREFIX, 8)
+    gx, gw = lbp.lbp_backward(x.to(dev), gy.to(dev), w.to(dev), 8, bases, gw_dtype=torch.bfloat16)
+    assert gw.dtype == torch.bfloat16
+    ox, ow = O.backward_lowrank(f64(x), f64(gy), f64(w), 8, bases)
+    assert rel(gx, ox) <= 2e-2 and rel(gw, ow) <= 2e-2
+
+
+def test_bf16_full_rank_is_exact_bp(dev):
+    case = synth.config_cases(3)[1]
+    x, gy, w = _inputs(3, 1, 16)
+    ex, ew = O.backward_exact(f64(x), f64(gy), f64(w))
+    for entry in (False, True):
+        _, _, gx, gw = _run_backward(dev, case, 64, batch=16, fullrank_entry=entry)
+        assert rel(gx, ex) <= 2e-2 and rel(gw, ew) <= 2e-2
+
+
+@pytest.mark.parametrize("idx,ranks", [(0, (1, 4, 7, 16)), (1, (1, 8, 21, 36)), (2, (1, 10, 36, 100))])
+def test_config5_sweep_full_size(dev, idx, ranks):
+    case = synth.config_cases(5)[idx]
+    for r in ranks:
+        _check_lowrank(dev, case, r)
+
+
+def test_outputs_do_not_depend_on_basis_order(dev):
+    case = synth.config_cases(3)[1]
+    x, gy, w = _inputs(3, 1, 4)
+    bases = O.select_bases(8, O.RULE_L1, 3)
+    perm = [bases[i] for i in (3, 0, 5, 1, 4, 2)]
+    a = lbp.lbp_backward(x.to(dev), gy.to(dev), w.to(dev), 8, bases)
+    b = lbp.lbp_backward(x.to(dev), gy.to(dev), w.to(dev), 8, perm)
+    assert rel(a[0], f64(b[0])) <= 1e-2 and rel(a[1], f64(b[1])) <= 1e-2
+
+
+def test_repeated_calls_are_deterministic(dev):
+    case = synth.config_cases(3)[1]
+    x, gy, w = _inputs(3, 1, 8)
+    bases = O.select_bases(8, O.RULE_PREFIX, 8)
+    xd, gd, wd = x.to(dev), gy.to(dev), w.to(dev)
+    a = lbp.lbp_backward(xd, gd, wd, 8, bases)
+    b = lbp.lbp_backward(xd, gd, wd, 8, bases)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
