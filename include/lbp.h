@@ -155,6 +155,25 @@ int lbp_backward_fullrank(const void* x, const void* g_y, const void* W,
  * LBP_ERR_CUDA. */
 int lbp_poll_status(void* ws, void* stream);
 
+/* ---- measurement hooks (no effect on results) ---------------------------- */
+
+/* Number of kernels this library has launched from the calling thread since it
+ * was loaded (a running count; take differences). */
+long long lbp_launch_count(void);
+
+/* Phase timing.  `events` is a HOST array of n cudaEvent_t handles (as void*),
+ * or NULL to switch the hook off; the setting is per calling thread and the
+ * array must stay valid while it is set.  While set, lbp_backward records
+ * events[0] on `stream` before its first kernel and events[i] after phase i
+ * (i < n), so that the elapsed time between events[i-1] and events[i] is the
+ * device time of phase i of Algorithm 1:
+ *   1 project x   2 project g_y   3 g_W product   4 g_x_hat product   5 expand
+ * (the full-rank mode records 0, 3 and 4 only).  lbp_phase_count() is the
+ * number of events a call may record, lbp_phase_name(i) a short label. */
+int lbp_set_phase_events(void** events, int n);
+int lbp_phase_count(void);
+const char* lbp_phase_name(int phase);
+
 #ifdef __cplusplus
 }
 #endif

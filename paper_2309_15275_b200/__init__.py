@@ -7,5 +7,6 @@ from .binding import (  # noqa: F401
     LBP_BF16, LBP_F32, SEL_L1, SEL_LINF, SEL_PREFIX, EXPORTED, LIB_PATH, LbpError,
     alloc_workspace, lbp_backward, lbp_backward_fullrank, lbp_basis_matrix, lbp_expand,
     lbp_flops, lbp_poll_status, lbp_project, lbp_select_bases, lbp_status_bytes,
-    lbp_status_string, lbp_workspace_bytes,
+    lbp_status_string, lbp_workspace_bytes, lbp_launch_count, lbp_phase_count, lbp_phase_name,
+    lbp_set_phase_events,
 )

@@ -77,13 +77,22 @@ def _lib() -> C.CDLL:
         lib.lbp_backward_fullrank.restype = i32
         lib.lbp_poll_status.argtypes = [vp, vp]
         lib.lbp_poll_status.restype = i32
+        lib.lbp_launch_count.argtypes = []
+        lib.lbp_launch_count.restype = C.c_longlong
+        lib.lbp_set_phase_events.argtypes = [C.POINTER(vp), i32]
+        lib.lbp_set_phase_events.restype = i32
+        lib.lbp_phase_count.argtypes = []
+        lib.lbp_phase_count.restype = i32
+        lib.lbp_phase_name.argtypes = [i32]
+        lib.lbp_phase_name.restype = C.c_char_p
         _LIB = lib
     return _LIB
 
 
 EXPORTED = ("lbp_select_bases", "lbp_basis_matrix", "lbp_flops", "lbp_status_string",
             "lbp_last_cuda_error", "lbp_workspace_bytes", "lbp_status_bytes", "lbp_project",
-            "lbp_expand", "lbp_backward", "lbp_backward_fullrank", "lbp_poll_status")
+            "lbp_expand", "lbp_backward", "lbp_backward_fullrank", "lbp_poll_status",
+            "lbp_launch_count", "lbp_set_phase_events", "lbp_phase_count", "lbp_phase_name")
 
 
 def _check(status: int, where: str) -> None:
@@ -242,3 +251,32 @@ def lbp_backward_fullrank(x, g_y, W, k: int, *, gw_dtype: torch.dtype = torch.fl
 def lbp_poll_status(ws: torch.Tensor) -> int:
     """Synchronises the current stream and returns the device status (0 = ok)."""
     return int(_lib().lbp_poll_status(_dev(ws, "ws"), _stream()))
+
+
+# ------------------------------------------------------ measurement hooks ----
+def lbp_launch_count() -> int:
+    return int(_lib().lbp_launch_count())
+
+
+def lbp_phase_count() -> int:
+    return int(_lib().lbp_phase_count())
+
+
+def lbp_phase_name(i: int) -> str:
+    return _lib().lbp_phase_name(i).decode()
+
+
+_PHASE_KEEPALIVE = None
+
+
+def lbp_set_phase_events(events) -> None:
+    """events: list of torch.cuda.Event (already created with enable_timing=True
+    and recorded once so their handles exist), or None to switch the hook off."""
+    global _PHASE_KEEPALIVE
+    if events is None:
+        _check(_lib().lbp_set_phase_events(None, 0), "lbp_set_phase_events")
+        _PHASE_KEEPALIVE = None
+        return
+    arr = (C.c_void_p * len(events))(*[e.cuda_event for e in events])
+    _check(_lib().lbp_set_phase_events(arr, len(events)), "lbp_set_phase_events")
+    _PHASE_KEEPALIVE = (arr, list(events))

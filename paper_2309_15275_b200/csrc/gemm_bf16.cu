@@ -362,6 +362,7 @@ int launch_gemm(const void* A, bool a_mn_major, const void* Bm, void* D, int in_
     }
     gemm_bf16_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(tmap_a, tmap_b, p);
   }
+  count_launch();
   LBP_CUDA_TRY(cudaGetLastError());
 
   if (t.splits > 1) {
@@ -369,6 +370,7 @@ int launch_gemm(const void* A, bool a_mn_major, const void* Bm, void* D, int in_
     const long long threads = (mn + 3) / 4;
     splitk_reduce_kernel<<<static_cast<unsigned>((threads + 255) / 256), 256, 0, stream>>>(
         splitk_ws, D, mn, t.splits, d_dtype == LBP_BF16 ? 1 : 0);
+    count_launch();
     LBP_CUDA_TRY(cudaGetLastError());
   }
   return LBP_OK;

@@ -86,6 +86,7 @@ int launch_gemm_fp32(const float* A, bool a_mn_major, const float* Bm, float* D,
     gemm_fp32_kernel<true><<<grid, 256, 0, stream>>>(A, Bm, D, M, N, K);
   else
     gemm_fp32_kernel<false><<<grid, 256, 0, stream>>>(A, Bm, D, M, N, K);
+  count_launch();
   LBP_CUDA_TRY(cudaGetLastError());
   return LBP_OK;
 }

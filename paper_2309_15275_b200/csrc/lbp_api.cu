@@ -139,19 +139,34 @@ static Layout plan_layout(const lbp_layer& L, int r) {
   return w;
 }
 
+// Phase-event hook (see lbp_set_phase_events).
+static thread_local void** g_phase_events = nullptr;
+static thread_local int g_phase_n = 0;
+constexpr int kPhaseCount = 6;
+
+static int mark_phase(int i, cudaStream_t stream) {
+  if (g_phase_events != nullptr && i < g_phase_n && g_phase_events[i] != nullptr)
+    LBP_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(g_phase_events[i]), stream));
+  return LBP_OK;
+}
+
 static int run_fullrank(const void* x, const void* g_y, const void* W, void* g_x, void* g_W,
                         const lbp_layer& L, uint8_t* ws, cudaStream_t stream) {
   const Layout lay = plan_layout(L, L.k * L.k);
   const long long T = lay.rows;
   uint32_t* status = reinterpret_cast<uint32_t*>(ws);
   float* sk = reinterpret_cast<float*>(ws + lay.splitk);
+  if (int e = mark_phase(0, stream)) return e;
   // Eq. 2: g_W = g_y^T x
   if (int e = launch_gemm(g_y, /*a_mn_major=*/true, x, g_W, L.dtype, L.gw_dtype, L.Cout, L.Cin, T,
                           sk, lay.splitk_bytes, status, stream))
     return e;
+  if (int e = mark_phase(3, stream)) return e;
   // Eq. 2: g_x = g_y W
-  return launch_gemm(g_y, /*a_mn_major=*/false, W, g_x, L.dtype, L.dtype, T, L.Cin, L.Cout, sk,
-                     lay.splitk_bytes, status, stream);
+  if (int e = launch_gemm(g_y, /*a_mn_major=*/false, W, g_x, L.dtype, L.dtype, T, L.Cin, L.Cout,
+                          sk, lay.splitk_bytes, status, stream))
+    return e;
+  return mark_phase(4, stream);
 }
 
 }  // namespace lbp
@@ -218,21 +233,29 @@ int lbp_backward(const void* x, const void* g_y, const void* W, void* g_x, void*
   float* sk = reinterpret_cast<float*>(wsb + lay.splitk);
   const RowMap dense{1, r};
 
+  if (int e = mark_phase(0, st)) return e;
   // Algorithm 1, steps 1-2: x_hat = p(x), g_y_hat = p(g_y)
   if (int e = launch_project(x, x_hat, L.dtype, L.B, L.H, L.W, L.Cin, plan, dense, status, st))
     return e;
+  if (int e = mark_phase(1, st)) return e;
   if (int e = launch_project(g_y, gy_hat, L.dtype, L.B, L.H, L.W, L.Cout, plan, dense, status, st))
     return e;
+  if (int e = mark_phase(2, st)) return e;
   // step 3: g_W = g_y_hat^T x_hat
   if (int e = launch_gemm(gy_hat, /*a_mn_major=*/true, x_hat, g_W, L.dtype, L.gw_dtype, L.Cout,
                           L.Cin, lay.rows, sk, lay.splitk_bytes, status, st))
     return e;
+  if (int e = mark_phase(3, st)) return e;
   // step 4: g_x_hat = g_y_hat W   (kept in fp32)
   if (int e = launch_gemm(gy_hat, /*a_mn_major=*/false, W, gx_hat, L.dtype, LBP_F32, lay.rows,
                           L.Cin, L.Cout, sk, lay.splitk_bytes, status, st))
     return e;
+  if (int e = mark_phase(4, st)) return e;
   // step 5: g_x = p^-1(g_x_hat)
-  return launch_expand(gx_hat, /*in_f32=*/true, g_x, L.dtype, L.B, L.H, L.W, L.Cin, plan, dense, st);
+  if (int e = launch_expand(gx_hat, /*in_f32=*/true, g_x, L.dtype, L.B, L.H, L.W, L.Cin, plan,
+                            dense, st))
+    return e;
+  return mark_phase(5, st);
 }
 
 int lbp_backward_fullrank(const void* x, const void* g_y, const void* W, void* g_x, void* g_W,
@@ -248,6 +271,27 @@ int lbp_backward_fullrank(const void* x, const void* g_y, const void* W, void* g
   if (int e = check_device_arch()) return e;
   return run_fullrank(x, g_y, W, g_x, g_W, *layer, static_cast<uint8_t*>(ws),
                       static_cast<cudaStream_t>(stream));
+}
+
+int lbp_set_phase_events(void** events, int n) {
+  if (events != nullptr && n < 1) return LBP_ERR_SHAPE;
+  g_phase_events = events;
+  g_phase_n = events ? n : 0;
+  return LBP_OK;
+}
+
+int lbp_phase_count(void) { return kPhaseCount; }
+
+const char* lbp_phase_name(int phase) {
+  switch (phase) {
+    case 0: return "start";
+    case 1: return "project_x";
+    case 2: return "project_gy";
+    case 3: return "gw_product";
+    case 4: return "gxhat_product";
+    case 5: return "expand";
+    default: return "";
+  }
 }
 
 int lbp_poll_status(void* ws, void* stream) {

@@ -12,6 +12,9 @@ namespace lbp {
 static thread_local int g_last_cuda_error = 0;
 void set_last_cuda_error(cudaError_t e) { g_last_cuda_error = static_cast<int>(e); }
 
+thread_local long long g_launches = 0;
+void count_launch(int n) { g_launches += n; }
+
 int check_order(int k) { return (k == 4 || k == 8 || k == 16) ? LBP_OK : LBP_ERR_BLOCK; }
 
 static int log2_int(int n) {
@@ -169,6 +172,8 @@ const char* lbp_status_string(int status) {
 }
 
 int lbp_last_cuda_error(void) { return g_last_cuda_error; }
+
+long long lbp_launch_count(void) { return lbp::g_launches; }
 
 size_t lbp_status_bytes(void) { return kStatusBytes; }
 

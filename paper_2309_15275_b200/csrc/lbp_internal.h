@@ -48,6 +48,7 @@ int walsh_sign(int k, int s, int u);
 int check_order(int k);
 
 void set_last_cuda_error(cudaError_t e);
+void count_launch(int n = 1);   // bumps the per-thread kernel-launch counter
 #define LBP_CUDA_TRY(expr)                       \
   do {                                           \
     cudaError_t e__ = (expr);                    \

@@ -158,6 +158,7 @@ static int launch_one(const TI* t_hat, TO* t, const ExpandParams& p, const Devic
   const long long cap = static_cast<long long>(sms) * 8;
   const int grid = static_cast<int>(want < cap ? want : cap);
   wht_expand_kernel<TI, TO, K, LB><<<grid, 256, 0, stream>>>(t_hat, t, p, plan);
+  count_launch();
   LBP_CUDA_TRY(cudaGetLastError());
   return LBP_OK;
 }

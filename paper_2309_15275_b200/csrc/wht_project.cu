@@ -222,6 +222,7 @@ static int launch_one(const CUtensorMap& tmap, T* out, const ProjParams& p, cons
   long long want = (p.n_items + Cfg::kWarps - 1) / Cfg::kWarps;
   const int grid = static_cast<int>(want < sms ? want : sms);
   kern<<<grid, Cfg::kWarps * 32, Cfg::kSmemBytes, stream>>>(tmap, out, p, plan);
+  count_launch();
   LBP_CUDA_TRY(cudaGetLastError());
   return LBP_OK;
 }

@@ -21,7 +21,7 @@ def _built():
 
 def test_library_exports_every_declared_symbol():
     header = open(os.path.join(ROOT, "include", "lbp.h")).read()
-    declared = set(re.findall(r"^(?:int|size_t|double|const char\*)\s+(lbp_[a-z_]+)\s*\(", header, re.M))
+    declared = set(re.findall(r"^(?:int|size_t|double|long long|const char\*)\s+(lbp_[a-z_]+)\s*\(", header, re.M))
     assert declared == set(lbp.EXPORTED)
     lib = ctypes.CDLL(lbp.LIB_PATH)
     for name in declared:
