@@ -167,7 +167,8 @@ long long lbp_launch_count(void);
  * events[0] on `stream` before its first kernel and events[i] after phase i
  * (i < n), so that the elapsed time between events[i-1] and events[i] is the
  * device time of phase i of Algorithm 1:
- *   1 project x   2 project g_y   3 g_W product   4 g_x_hat product   5 expand
+ *   1 project x and g_y (one launch)   2 (unused, recorded with 1)
+ *   3 g_W product   4 g_x_hat product   5 expand
  * (the full-rank mode records 0, 3 and 4 only).  lbp_phase_count() is the
  * number of events a call may record, lbp_phase_name(i) a short label. */
 int lbp_set_phase_events(void** events, int n);

@@ -44,7 +44,7 @@ static int get_encode_fn(EncodeTiledFn* out) {
 }
 
 int encode_block_tensor_map(CUtensorMap* map, const void* base, int dtype, int B, int H, int W,
-                            int C, int k, int box_c) {
+                            int C, int k, int box_c, bool swizzle128) {
   EncodeTiledFn enc;
   if (int e = get_encode_fn(&enc)) return e;
   const cuuint64_t es = static_cast<cuuint64_t>(elem_size(dtype));
@@ -58,7 +58,8 @@ int encode_block_tensor_map(CUtensorMap* map, const void* base, int dtype, int B
   const CUresult r =
       enc(map, dtype == LBP_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
           4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-          CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+          CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     set_last_cuda_error(cudaErrorInvalidValue);
@@ -234,12 +235,11 @@ int lbp_backward(const void* x, const void* g_y, const void* W, void* g_x, void*
   const RowMap dense{1, r};
 
   if (int e = mark_phase(0, st)) return e;
-  // Algorithm 1, steps 1-2: x_hat = p(x), g_y_hat = p(g_y)
-  if (int e = launch_project(x, x_hat, L.dtype, L.B, L.H, L.W, L.Cin, plan, dense, status, st))
+  // Algorithm 1, steps 1-2: x_hat = p(x), g_y_hat = p(g_y), one launch for both
+  if (int e = launch_project2(g_y, gy_hat, L.Cout, x, x_hat, L.Cin, L.dtype, L.B, L.H, L.W, plan,
+                              dense, status, st))
     return e;
   if (int e = mark_phase(1, st)) return e;
-  if (int e = launch_project(g_y, gy_hat, L.dtype, L.B, L.H, L.W, L.Cout, plan, dense, status, st))
-    return e;
   if (int e = mark_phase(2, st)) return e;
   // step 3: g_W = g_y_hat^T x_hat
   if (int e = launch_gemm(gy_hat, /*a_mn_major=*/true, x_hat, g_W, L.dtype, L.gw_dtype, L.Cout,
@@ -285,8 +285,8 @@ int lbp_phase_count(void) { return kPhaseCount; }
 const char* lbp_phase_name(int phase) {
   switch (phase) {
     case 0: return "start";
-    case 1: return "project_x";
-    case 2: return "project_gy";
+    case 1: return "project_x_gy";
+    case 2: return "unused";
     case 3: return "gw_product";
     case 4: return "gxhat_product";
     case 5: return "expand";

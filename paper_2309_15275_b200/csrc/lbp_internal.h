@@ -35,6 +35,10 @@ struct BasisPlan {
   int32_t r;
   int32_t LB;
   int16_t qmap[kMaxRank];  // [a * LB + b]
+  // order-k natural (Sylvester) row indices of the selected Walsh rows:
+  // wal_{i_q}[u] = (-1)^popcount(nat_i[q] & u), likewise for j along W
+  uint8_t nat_i[kMaxRank];
+  uint8_t nat_j[kMaxRank];
 };
 
 // Validates (k, set, r) and fills `plan`.  Returns an lbp_status.
@@ -60,9 +64,9 @@ void count_launch(int n = 1);   // bumps the per-thread kernel-launch counter
 
 // ---- tensor maps (TMA descriptors), encoded on the host ------------------
 // 4-D channels-last tensor (B, H, W, C): box = one k x k block x box_c
-// channels, no swizzle.
+// channels; no swizzle, or the 128-byte swizzle (box_c * element size must be 128).
 int encode_block_tensor_map(CUtensorMap* map, const void* base, int dtype, int B, int H, int W,
-                            int C, int k, int box_c);
+                            int C, int k, int box_c, bool swizzle128);
 // 2-D row-major bf16 matrix (rows, cols): box = box_rows x 64 columns (128 B),
 // 128-byte swizzle.
 int encode_matrix_tensor_map(CUtensorMap* map, const void* base, long long rows, long long cols,
@@ -78,6 +82,11 @@ struct RowMap {
 
 int launch_project(const void* t, void* t_hat, int dtype, int B, int H, int W, int C,
                    const BasisPlan& plan, RowMap rows, uint32_t* status, cudaStream_t stream);
+
+// Projects two tensors that share the token grid (x and g_y) in one launch.
+int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* out1, int C1,
+                    int dtype, int B, int H, int W, const BasisPlan& plan, RowMap rows,
+                    uint32_t* status, cudaStream_t stream);
 
 // t_hat is fp32 when `in_f32`, else of `dtype`; t is of `dtype`.
 int launch_expand(const void* t_hat, bool in_f32, void* t, int dtype, int B, int H, int W, int C,

@@ -10,24 +10,9 @@
 #include "lbp_internal.h"
 #include "ptx_sm100.cuh"
 #include "wht_device.cuh"
+#include "wht_project.cuh"
 
 namespace lbp {
-
-struct ProjParams {
-  int32_t nb, Hb, Wb, C, r, n_chunks;
-  int32_t bpt, tile_rows;
-  long long n_items;   // nb * n_chunks
-  uint32_t* status;
-  float scale;         // 1/k
-};
-
-template <int K, bool BF16>
-struct ProjCfg {
-  static constexpr int kTileBytesMax = K * K * 128;
-  static constexpr int kWarps = (K == 16) ? 6 : 12;
-  static constexpr int kStages = (K == 4) ? 4 : (K == 8 ? 2 : 1);
-  static constexpr int kSmemBytes = kWarps * kStages * kTileBytesMax + kWarps * kStages * 8 + 128;
-};
 
 template <typename T, bool BF16, int NCH>
 __device__ __forceinline__ void store_coeff(T* __restrict__ out, long long row, int C, int c0,
@@ -43,8 +28,9 @@ __device__ __forceinline__ void store_coeff(T* __restrict__ out, long long row, 
 
 template <typename T, int K, int LB>
 __global__ void __launch_bounds__(ProjCfg<K, sizeof(T) == 2>::kWarps * 32, 1)
-    wht_project_kernel(const __grid_constant__ CUtensorMap tmap, T* __restrict__ out,
-                       const __grid_constant__ ProjParams p,
+    wht_project_kernel(const __grid_constant__ CUtensorMap tmap0,
+                       const __grid_constant__ CUtensorMap tmap1, T* __restrict__ out0,
+                       T* __restrict__ out1, const __grid_constant__ ProjParams p,
                        const __grid_constant__ DevicePlan plan) {
   constexpr bool BF16 = sizeof(T) == 2;
   using Cfg = ProjCfg<K, BF16>;
@@ -65,41 +51,51 @@ __global__ void __launch_bounds__(ProjCfg<K, sizeof(T) == 2>::kWarps * 32, 1)
     for (int s = 0; s < S; ++s) ptx::mbar_init(&my_bars[s], 1);
     ptx::mbar_fence_init();
   }
-  if (threadIdx.x == 0) ptx::prefetch_tensormap(&tmap);
+  if (threadIdx.x == 0) {
+    ptx::prefetch_tensormap(&tmap0);
+    ptx::prefetch_tensormap(&tmap1);
+  }
   __syncthreads();
 
-  const long long first = static_cast<long long>(blockIdx.x) * NW + warp;
-  const long long stride = static_cast<long long>(gridDim.x) * NW;
-  const long long n_my = first < p.n_items ? (p.n_items - first + stride - 1) / stride : 0;
+  const uint32_t first = blockIdx.x * NW + warp;
+  const uint32_t stride = gridDim.x * NW;
+  const uint32_t n_my = first < p.n_items ? (p.n_items - first + stride - 1) / stride : 0;
   constexpr int ch_per_tile = 32 * CH_PER_WORD;   // a token is 128 B = 32 words wide in a tile
   constexpr int tw = 32;
 
-  auto issue = [&](long long idx, int s) {
-    const long long item = first + idx * stride;
-    const int chunk = static_cast<int>(item % p.n_chunks);
-    const int blk = static_cast<int>(item / p.n_chunks);
-    const int bw = blk % p.Wb, bh = (blk / p.Wb) % p.Hb, b = blk / (p.Wb * p.Hb);
+  auto issue = [&](uint32_t idx, int s) {
+    uint32_t item = first + idx * stride;
+    const int which = item >= p.n_items0;
+    if (which) item -= p.n_items0;
+    const uint32_t nch = static_cast<uint32_t>(p.n_chunks[which]);
+    const uint32_t blk = item / nch, chunk = item - blk * nch;
+    const uint32_t bw = blk % p.Wb, t2 = blk / p.Wb, bh = t2 % p.Hb, b = t2 / p.Hb;
     ptx::mbar_expect_tx(&my_bars[s], static_cast<uint32_t>(Cfg::kTileBytesMax));
-    ptx::tma_load_4d(my_tiles + s * Cfg::kTileBytesMax, &tmap, &my_bars[s], chunk * ch_per_tile,
-                     bw * K, bh * K, b);
+    ptx::tma_load_4d(my_tiles + s * Cfg::kTileBytesMax, which ? &tmap1 : &tmap0, &my_bars[s],
+                     chunk * ch_per_tile, bw * K, bh * K, b);
   };
 
   if (lane == 0) {
-    for (int i = 0; i < S && i < n_my; ++i) issue(i, i);
+    for (uint32_t i = 0; i < S && i < n_my; ++i) issue(i, i);
   }
 
-  for (long long idx = 0; idx < n_my; ++idx) {
+  for (uint32_t idx = 0; idx < n_my; ++idx) {
     const int s = static_cast<int>(idx % S);
-    const uint32_t parity = static_cast<uint32_t>((idx / S) & 1);
+    const uint32_t parity = (idx / S) & 1u;
     const bool ok = ptx::mbar_wait(&my_bars[s], parity, p.status, (1u << 16) | 1u);
     if (!__all_sync(0xffffffffu, ok)) break;
 
-    const long long item = first + idx * stride;
-    const int chunk = static_cast<int>(item % p.n_chunks);
-    const int blk = static_cast<int>(item / p.n_chunks);
+    uint32_t item = first + idx * stride;
+    const int which = item >= p.n_items0;
+    if (which) item -= p.n_items0;
+    const uint32_t nch = static_cast<uint32_t>(p.n_chunks[which]);
+    const int blk = static_cast<int>(item / nch);
+    const int chunk = static_cast<int>(item - blk * nch);
+    const int C = p.C[which];
+    T* __restrict__ out = which ? out1 : out0;
     const uint32_t* tile = reinterpret_cast<const uint32_t*>(my_tiles + s * Cfg::kTileBytesMax);
     const int c0 = chunk * ch_per_tile + lane * CH_PER_WORD;
-    const bool active = c0 < p.C;   // channels past C are zero-filled by TMA and skipped
+    const bool active = c0 < C;   // channels past C are zero-filled by TMA and skipped
     const long long row0 =
         static_cast<long long>(blk / p.bpt) * p.tile_rows + static_cast<long long>(blk % p.bpt) * p.r;
 
@@ -136,7 +132,7 @@ __global__ void __launch_bounds__(ProjCfg<K, sizeof(T) == 2>::kWarps * 32, 1)
 #pragma unroll
             for (int b = 0; b < LB; ++b) {
               const int q = plan.qmap[a * LB + b];
-              if (q >= 0) store_coeff<T, BF16, NCH>(out, row0 + q, p.C, c0, pass, acc[a][b], p.scale);
+              if (q >= 0) store_coeff<T, BF16, NCH>(out, row0 + q, C, c0, pass, acc[a][b], p.scale);
             }
           }
         }
@@ -180,7 +176,7 @@ __global__ void __launch_bounds__(ProjCfg<K, sizeof(T) == 2>::kWarps * 32, 1)
                 const int q = plan.qmap[a * 16 + nh * 4 + n_lo];
                 if (q >= 0) {
                   const float v1[1] = {R[nh][a]};
-                  store_coeff<T, BF16, 1>(out, row0 + q, p.C, c0, pass, v1, p.scale);
+                  store_coeff<T, BF16, 1>(out, row0 + q, C, c0, pass, v1, p.scale);
                 }
               }
             }
@@ -192,9 +188,9 @@ __global__ void __launch_bounds__(ProjCfg<K, sizeof(T) == 2>::kWarps * 32, 1)
         const long long tile_base = static_cast<long long>(blk / p.bpt) * p.tile_rows;
         for (long long row = row0 + p.r; row < tile_base + p.tile_rows; ++row) {
           if constexpr (BF16) {
-            *reinterpret_cast<uint32_t*>(out + row * p.C + c0) = 0u;
+            *reinterpret_cast<uint32_t*>(out + row * C + c0) = 0u;
           } else {
-            out[row * p.C + c0] = 0.f;
+            out[row * C + c0] = 0.f;
           }
         }
       }
@@ -209,84 +205,116 @@ __global__ void __launch_bounds__(ProjCfg<K, sizeof(T) == 2>::kWarps * 32, 1)
 }
 
 template <typename T, int K, int LB>
-static int launch_one(const CUtensorMap& tmap, T* out, const ProjParams& p, const DevicePlan& plan,
-                      int sms, cudaStream_t stream) {
+static int launch_one(const CUtensorMap* tmaps, T* out0, T* out1, const ProjParams& p,
+                      const DevicePlan& plan, int sms, cudaStream_t stream) {
   using Cfg = ProjCfg<K, sizeof(T) == 2>;
   auto kern = wht_project_kernel<T, K, LB>;
-  static bool configured = false;
-  if (!configured) {
+  static bool configured[64] = {};
+  int dev = 0;
+  LBP_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
     LBP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       Cfg::kSmemBytes));
-    configured = true;
+    if (dev >= 0 && dev < 64) configured[dev] = true;
   }
-  long long want = (p.n_items + Cfg::kWarps - 1) / Cfg::kWarps;
-  const int grid = static_cast<int>(want < sms ? want : sms);
-  kern<<<grid, Cfg::kWarps * 32, Cfg::kSmemBytes, stream>>>(tmap, out, p, plan);
+  const uint32_t want = (p.n_items + Cfg::kWarps - 1) / Cfg::kWarps;
+  const int grid = static_cast<int>(want < static_cast<uint32_t>(sms) ? want : sms);
+  kern<<<grid, Cfg::kWarps * 32, Cfg::kSmemBytes, stream>>>(tmaps[0], tmaps[1], out0, out1, p, plan);
   count_launch();
   LBP_CUDA_TRY(cudaGetLastError());
   return LBP_OK;
 }
 
 template <typename T, int K>
-static int launch_k(int LB, const CUtensorMap& tmap, T* out, const ProjParams& p,
+static int launch_k(int LB, const CUtensorMap* tmaps, T* out0, T* out1, const ProjParams& p,
                     const DevicePlan& plan, int sms, cudaStream_t stream) {
   switch (LB) {
-    case 1: return launch_one<T, K, 1>(tmap, out, p, plan, sms, stream);
-    case 2: return launch_one<T, K, 2>(tmap, out, p, plan, sms, stream);
-    case 4: return launch_one<T, K, 4>(tmap, out, p, plan, sms, stream);
+    case 1: return launch_one<T, K, 1>(tmaps, out0, out1, p, plan, sms, stream);
+    case 2: return launch_one<T, K, 2>(tmaps, out0, out1, p, plan, sms, stream);
+    case 4: return launch_one<T, K, 4>(tmaps, out0, out1, p, plan, sms, stream);
     case 8:
-      if constexpr (K >= 8) return launch_one<T, K, 8>(tmap, out, p, plan, sms, stream);
+      if constexpr (K >= 8) return launch_one<T, K, 8>(tmaps, out0, out1, p, plan, sms, stream);
       break;
     case 16:
-      if constexpr (K >= 16) return launch_one<T, K, 16>(tmap, out, p, plan, sms, stream);
+      if constexpr (K >= 16) return launch_one<T, K, 16>(tmaps, out0, out1, p, plan, sms, stream);
       break;
   }
   return LBP_ERR_BASIS;
 }
 
 template <typename T>
-static int launch_t(const CUtensorMap& tmap, T* out, const ProjParams& p, const BasisPlan& bp,
-                    const DevicePlan& plan, int sms, cudaStream_t stream) {
+static int launch_t(const CUtensorMap* tmaps, T* out0, T* out1, const ProjParams& p,
+                    const BasisPlan& bp, const DevicePlan& plan, int sms, cudaStream_t stream) {
   switch (bp.k) {
-    case 4: return launch_k<T, 4>(bp.LB, tmap, out, p, plan, sms, stream);
-    case 8: return launch_k<T, 8>(bp.LB, tmap, out, p, plan, sms, stream);
-    case 16: return launch_k<T, 16>(bp.LB, tmap, out, p, plan, sms, stream);
+    case 4: return launch_k<T, 4>(bp.LB, tmaps, out0, out1, p, plan, sms, stream);
+    case 8: return launch_k<T, 8>(bp.LB, tmaps, out0, out1, p, plan, sms, stream);
+    case 16: return launch_k<T, 16>(bp.LB, tmaps, out0, out1, p, plan, sms, stream);
   }
   return LBP_ERR_BLOCK;
 }
 
-int launch_project(const void* t, void* t_hat, int dtype, int B, int H, int W, int C,
-                   const BasisPlan& bp, RowMap rows, uint32_t* status, cudaStream_t stream) {
+int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* out1, int C1,
+                    int dtype, int B, int H, int W, const BasisPlan& bp, RowMap rows,
+                    uint32_t* status, cudaStream_t stream) {
   const int K = bp.k;
   const int es = dtype == LBP_BF16 ? 2 : 4;
   const int box_c = 128 / es;   // a box wider than C is legal: the excess is zero-filled
 
-  CUtensorMap tmap;
-  if (int e = encode_block_tensor_map(&tmap, t, dtype, B, H, W, C, K, box_c)) return e;
+  CUtensorMap tmaps[2];
+  if (int e = encode_block_tensor_map(&tmaps[0], t0, dtype, B, H, W, C0, K, box_c, false)) return e;
+  if (t1 != nullptr) {
+    if (int e = encode_block_tensor_map(&tmaps[1], t1, dtype, B, H, W, C1, K, box_c, false)) return e;
+  } else {
+    tmaps[1] = tmaps[0];
+  }
 
   ProjParams p;
   p.Hb = H / K;
   p.Wb = W / K;
   p.nb = B * p.Hb * p.Wb;
-  p.C = C;
   p.r = bp.r;
-  p.n_chunks = (C + box_c - 1) / box_c;
   p.bpt = rows.bpt;
   p.tile_rows = rows.tile_rows;
-  p.n_items = static_cast<long long>(p.nb) * p.n_chunks;
+  p.C[0] = C0;
+  p.C[1] = t1 ? C1 : C0;
+  p.n_chunks[0] = (C0 + box_c - 1) / box_c;
+  p.n_chunks[1] = t1 ? (C1 + box_c - 1) / box_c : 1;
+  const long long n0 = static_cast<long long>(p.nb) * p.n_chunks[0];
+  const long long n1 = t1 ? static_cast<long long>(p.nb) * p.n_chunks[1] : 0;
+  if (n0 + n1 >= (1ll << 31)) return LBP_ERR_SHAPE;
+  p.n_items0 = static_cast<uint32_t>(n0);
+  p.n_items = static_cast<uint32_t>(n0 + n1);
   p.status = status;
   p.scale = 1.0f / static_cast<float>(K);
-
-  DevicePlan plan;
-  for (int n = 0; n < 256; ++n) plan.qmap[n] = bp.qmap[n];
 
   int dev = 0, sms = 0;
   LBP_CUDA_TRY(cudaGetDevice(&dev));
   LBP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
 
+  if (dtype == LBP_BF16 && project_mma_supported(K, bp.r)) {
+    // bf16 data at moderate rank: the +-1 basis matrix is applied on the tensor pipe
+    CUtensorMap sw[2];
+    if (int e = encode_block_tensor_map(&sw[0], t0, dtype, B, H, W, C0, K, box_c, true)) return e;
+    sw[1] = sw[0];
+    if (t1 != nullptr)
+      if (int e = encode_block_tensor_map(&sw[1], t1, dtype, B, H, W, C1, K, box_c, true)) return e;
+    return launch_project_mma(sw, static_cast<__nv_bfloat16*>(out0),
+                              static_cast<__nv_bfloat16*>(out1), p, bp, sms, stream);
+  }
+
+  DevicePlan plan;
+  for (int n = 0; n < 256; ++n) plan.qmap[n] = bp.qmap[n];
+
   if (dtype == LBP_BF16)
-    return launch_t<__nv_bfloat16>(tmap, static_cast<__nv_bfloat16*>(t_hat), p, bp, plan, sms, stream);
-  return launch_t<float>(tmap, static_cast<float*>(t_hat), p, bp, plan, sms, stream);
+    return launch_t<__nv_bfloat16>(tmaps, static_cast<__nv_bfloat16*>(out0),
+                                   static_cast<__nv_bfloat16*>(out1), p, bp, plan, sms, stream);
+  return launch_t<float>(tmaps, static_cast<float*>(out0), static_cast<float*>(out1), p, bp, plan,
+                         sms, stream);
+}
+
+int launch_project(const void* t, void* t_hat, int dtype, int B, int H, int W, int C,
+                   const BasisPlan& bp, RowMap rows, uint32_t* status, cudaStream_t stream) {
+  return launch_project2(t, t_hat, C, nullptr, nullptr, 0, dtype, B, H, W, bp, rows, status, stream);
 }
 
 }  // namespace lbp

@@ -1,0 +1,36 @@
+// Shared between the two projection kernels (additions-only and tensor-pipe).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "lbp_internal.h"
+
+namespace lbp {
+
+// One launch projects up to two tensors that share the token grid (x and g_y of
+// a layer): items [0, n_items0) belong to tensor 0, the rest to tensor 1.
+struct ProjParams {
+  int32_t nb, Hb, Wb, r;
+  int32_t bpt, tile_rows;
+  int32_t C[2], n_chunks[2];
+  uint32_t n_items0, n_items;   // nb * n_chunks[0], nb * (n_chunks[0] + n_chunks[1])
+  uint32_t* status;
+  float scale;                  // 1/k
+};
+
+template <int K, bool BF16>
+struct ProjCfg {
+  static constexpr int kTileBytesMax = K * K * 128;
+  static constexpr int kWarps = (K == 16) ? 6 : 12;
+  static constexpr int kStages = (K == 4) ? 4 : (K == 8 ? 2 : 1);
+  static constexpr int kSmemBytes = kWarps * kStages * kTileBytesMax + kWarps * kStages * 8 + 128;
+};
+
+// Tensor-pipe projection (bf16 data): supported ranks per order.
+bool project_mma_supported(int k, int r);
+int launch_project_mma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloat16* out1,
+                       const ProjParams& p, const BasisPlan& bp, int sms, cudaStream_t stream);
+
+}  // namespace lbp

@@ -1,0 +1,262 @@
+// Projection kernel for bf16 data (Eq. 6 as the paper writes it: the block,
+// as a k*k x C matrix, times the k*k x r matrix of +-1 bases).
+//
+// The pass is HBM-bound; what has to stay small is the instruction count per
+// byte.  Applying the +-1 basis matrix with warp-level bf16 MMAs (exact
+// products, fp32 accumulation) needs about a quarter of the instructions of the
+// register butterfly, which keeps the load pipeline, not the issue slots, the
+// limiter.  Data movement is the same as in the additions-only kernel: one warp
+// owns a ring of shared-memory stages, lane 0 issues one 4-D TMA box per
+// (block, 64-channel chunk), here with the 128-byte swizzle so that ldmatrix
+// reads are conflict-free.
+//
+// Per tile:  D[q, c] = sum_tok A[q, tok] * X[tok, c]
+//   A (r rows padded to 16*MT, k*k columns) lives in registers for the whole
+//   kernel, X is the shared-memory tile (tokens x 64 channels), D is scaled by
+//   1/k, rounded once to bf16 and stored.
+#include <cuda_bf16.h>
+
+#include "lbp_internal.h"
+#include "ptx_sm100.cuh"
+#include "wht_device.cuh"
+#include "wht_project.cuh"
+
+namespace lbp {
+
+struct MmaPlan {
+  uint8_t nat_i[64];
+  uint8_t nat_j[64];
+};
+
+template <int K>
+struct MmaCfg {
+  static constexpr int kTokens = K * K;
+  static constexpr int kTileBytes = kTokens * 128;
+  static constexpr int kKSteps = kTokens / 16;
+  static constexpr int kWarps = (K == 16) ? 6 : 12;
+  static constexpr int kStages = (K == 4) ? 4 : (K == 8 ? 2 : 1);
+  static constexpr int kSmemBytes = kWarps * kStages * kTileBytes + kWarps * kStages * 8 + 1024;
+};
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1,
+                                                  uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr)
+               : "memory");
+}
+
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
+                                               uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 "
+      "{%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// bf16 bits of the basis entry B_{iq,jq}[tok] (+1, -1) or 0 for a padding row.
+template <int K>
+__device__ __forceinline__ uint32_t basis_bits(const MmaPlan& mp, int q, int r, int tok) {
+  if (q >= r) return 0u;
+  const int u = tok / K, v = tok % K;
+  const int neg = (__popc(mp.nat_i[q] & u) + __popc(mp.nat_j[q] & v)) & 1;
+  return neg ? 0xBF80u : 0x3F80u;
+}
+
+template <int K, int MT>
+__global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
+    wht_project_mma_kernel(const __grid_constant__ CUtensorMap tmap0,
+                           const __grid_constant__ CUtensorMap tmap1,
+                           __nv_bfloat16* __restrict__ out0, __nv_bfloat16* __restrict__ out1,
+                           const __grid_constant__ ProjParams p,
+                           const __grid_constant__ MmaPlan mp) {
+  using Cfg = MmaCfg<K>;
+  constexpr int NW = Cfg::kWarps, S = Cfg::kStages, KS = Cfg::kKSteps;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + NW * S * Cfg::kTileBytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, tq = lane & 3;
+  uint64_t* my_bars = bars + warp * S;
+  uint8_t* my_tiles = tiles + warp * S * Cfg::kTileBytes;
+
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < S; ++s) ptx::mbar_init(&my_bars[s], 1);
+    ptx::mbar_fence_init();
+  }
+  if (threadIdx.x == 0) {
+    ptx::prefetch_tensormap(&tmap0);
+    ptx::prefetch_tensormap(&tmap1);
+  }
+  __syncthreads();
+
+  const uint32_t first = blockIdx.x * NW + warp;
+  const uint32_t stride = gridDim.x * NW;
+  const uint32_t n_my = first < p.n_items ? (p.n_items - first + stride - 1) / stride : 0;
+
+  auto issue = [&](uint32_t idx, int s) {
+    uint32_t item = first + idx * stride;
+    const int which = item >= p.n_items0;
+    if (which) item -= p.n_items0;
+    const uint32_t nch = static_cast<uint32_t>(p.n_chunks[which]);
+    const uint32_t blk = item / nch, chunk = item - blk * nch;
+    const uint32_t bw = blk % p.Wb, t2 = blk / p.Wb, bh = t2 % p.Hb, b = t2 / p.Hb;
+    ptx::mbar_expect_tx(&my_bars[s], static_cast<uint32_t>(Cfg::kTileBytes));
+    ptx::tma_load_4d(my_tiles + s * Cfg::kTileBytes, which ? &tmap1 : &tmap0, &my_bars[s],
+                     chunk * 64, bw * K, bh * K, b);
+  };
+  if (lane == 0) {
+    for (uint32_t i = 0; i < S && i < n_my; ++i) issue(i, i);
+  }
+
+  // A fragments of m16n8k16, row-major: a0 (row g, k 2tq..+1), a1 (row g+8, same k),
+  // a2 (row g, k+8), a3 (row g+8, k+8); the low half of a register is the lower k.
+  uint32_t afrag[MT][KS][4];
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int q = mt * 16 + g + (j & 1) * 8;
+        const int tok = ks * 16 + 2 * tq + (j >> 1) * 8;
+        afrag[mt][ks][j] = basis_bits<K>(mp, q, p.r, tok) | (basis_bits<K>(mp, q, p.r, tok + 1) << 16);
+      }
+    }
+  }
+
+  // ldmatrix.x4.trans source rows: lane -> matrix (lane >> 3), row (lane & 7);
+  // matrices 0/1 are tokens +0..7 / +8..15 of channels 0..7 of a 16-channel pair,
+  // matrices 2/3 the same tokens of channels 8..15.
+  const int ld_tok = ((lane >> 3) & 1) * 8 + (lane & 7);
+  const int ld_chunk = lane >> 4;
+
+  for (uint32_t idx = 0; idx < n_my; ++idx) {
+    const int s = static_cast<int>(idx % S);
+    const uint32_t parity = (idx / S) & 1u;
+    const bool ok = ptx::mbar_wait(&my_bars[s], parity, p.status, (3u << 16) | 1u);
+    if (!__all_sync(0xffffffffu, ok)) break;
+
+    uint32_t item = first + idx * stride;
+    const int which = item >= p.n_items0;
+    if (which) item -= p.n_items0;
+    const uint32_t nch = static_cast<uint32_t>(p.n_chunks[which]);
+    const int blk = static_cast<int>(item / nch);
+    const int chunk = static_cast<int>(item - blk * nch);
+    const int C = p.C[which];
+    __nv_bfloat16* __restrict__ out = which ? out1 : out0;
+    const uint32_t tile = ptx::smem_u32(my_tiles + s * Cfg::kTileBytes);
+
+    float d[MT][8][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) d[mt][nt][j] = 0.f;
+
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      const int tok = ks * 16 + ld_tok;
+#pragma unroll
+      for (int np = 0; np < 4; ++np) {
+        const int c16 = np * 2 + ld_chunk;   // 16-byte chunk of the 128-byte token row
+        uint32_t b0, b1, b2, b3;
+        ldmatrix_x4_trans(tile + tok * 128 + ((c16 ^ (tok & 7)) << 4), b0, b1, b2, b3);
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          mma_bf16_16816(d[mt][2 * np], afrag[mt][ks], b0, b1);
+          mma_bf16_16816(d[mt][2 * np + 1], afrag[mt][ks], b2, b3);
+        }
+      }
+    }
+
+    // D fragment: d[0..1] = (row g, channels 2tq..+1), d[2..3] = (row g+8, same channels)
+    const long long row0 =
+        static_cast<long long>(blk / p.bpt) * p.tile_rows + static_cast<long long>(blk % p.bpt) * p.r;
+    const int cbase = chunk * 64 + 2 * tq;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+      const int q0 = mt * 16 + g, q1 = q0 + 8;
+#pragma unroll
+      for (int nt = 0; nt < 8; ++nt) {
+        const int c = cbase + nt * 8;
+        if (c < C) {   // C is a multiple of 8: a group of 8 channels is all in or all out
+          if (q0 < p.r)
+            *reinterpret_cast<uint32_t*>(out + (row0 + q0) * C + c) =
+                pack_bf16x2(d[mt][nt][0] * p.scale, d[mt][nt][1] * p.scale);
+          if (q1 < p.r)
+            *reinterpret_cast<uint32_t*>(out + (row0 + q1) * C + c) =
+                pack_bf16x2(d[mt][nt][2] * p.scale, d[mt][nt][3] * p.scale);
+        }
+      }
+    }
+    // rows of a padded row tile that no block owns are kept at zero
+    if (p.bpt > 1 && ((blk % p.bpt) == p.bpt - 1 || blk == p.nb - 1)) {
+      const long long tile_base = static_cast<long long>(blk / p.bpt) * p.tile_rows;
+      const int c = chunk * 64 + lane * 2;
+      if (c < C)
+        for (long long row = row0 + p.r; row < tile_base + p.tile_rows; ++row)
+          *reinterpret_cast<uint32_t*>(out + row * C + c) = 0u;
+    }
+
+    __syncwarp();
+    if (lane == 0 && idx + S < n_my) {
+      ptx::fence_proxy_async_smem();
+      issue(idx + S, s);
+    }
+  }
+}
+
+bool project_mma_supported(int k, int r) {
+  if (k == 4) return r <= 16;
+  if (k == 8) return r <= 32;
+  if (k == 16) return r <= 16;
+  return false;
+}
+
+template <int K, int MT>
+static int launch_mma_one(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloat16* out1,
+                          const ProjParams& p, const MmaPlan& mp, int sms, cudaStream_t stream) {
+  using Cfg = MmaCfg<K>;
+  auto kern = wht_project_mma_kernel<K, MT>;
+  static bool configured[64] = {};
+  int dev = 0;
+  LBP_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
+    LBP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      Cfg::kSmemBytes));
+    if (dev >= 0 && dev < 64) configured[dev] = true;
+  }
+  const uint32_t want = (p.n_items + Cfg::kWarps - 1) / Cfg::kWarps;
+  const int grid = static_cast<int>(want < static_cast<uint32_t>(sms) ? want : sms);
+  kern<<<grid, Cfg::kWarps * 32, Cfg::kSmemBytes, stream>>>(tmaps[0], tmaps[1], out0, out1, p, mp);
+  count_launch();
+  LBP_CUDA_TRY(cudaGetLastError());
+  return LBP_OK;
+}
+
+int launch_project_mma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloat16* out1,
+                       const ProjParams& p, const BasisPlan& bp, int sms, cudaStream_t stream) {
+  MmaPlan mp;
+  for (int q = 0; q < 64; ++q) {
+    mp.nat_i[q] = q < bp.r ? bp.nat_i[q] : 0;
+    mp.nat_j[q] = q < bp.r ? bp.nat_j[q] : 0;
+  }
+  const int mt = (bp.r + 15) / 16;
+  switch (bp.k) {
+    case 4: return launch_mma_one<4, 1>(tmaps, out0, out1, p, mp, sms, stream);
+    case 8:
+      if (mt == 1) return launch_mma_one<8, 1>(tmaps, out0, out1, p, mp, sms, stream);
+      return launch_mma_one<8, 2>(tmaps, out0, out1, p, mp, sms, stream);
+    case 16: return launch_mma_one<16, 1>(tmaps, out0, out1, p, mp, sms, stream);
+  }
+  return LBP_ERR_BLOCK;
+}
+
+}  // namespace lbp
