@@ -3,6 +3,9 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <cstdlib>
+
+#include "lbp_fused.cuh"
 #include "lbp_internal.h"
 
 namespace lbp {
@@ -107,9 +110,16 @@ static int check_layer(const lbp_layer* L) {
 
 // Workspace layout of lbp_backward at rank r < k*k.
 struct Layout {
-  size_t x_hat, gy_hat, gx_hat, splitk, splitk_bytes, total;
+  size_t x_hat, gy_hat, gx_hat, splitk, splitk_bytes, fused, total;
   long long rows;   // M_hat = blocks * r
 };
+
+// The persistent products kernel can be switched off (LBP_FUSED=0) to run the
+// separate product and expansion kernels instead.
+static bool fused_enabled() {
+  const char* e = std::getenv("LBP_FUSED");
+  return !(e != nullptr && e[0] == '0');
+}
 
 static Layout plan_layout(const lbp_layer& L, int r) {
   Layout w{};
@@ -136,6 +146,11 @@ static Layout plan_layout(const lbp_layer& L, int r) {
   }
   w.splitk = off = align_up(off, 1024);
   off += w.splitk_bytes;
+  // scratch of the persistent products kernel (bf16, k = 8, r <= 16): x_hat and
+  // g_y_hat with rows padded to 128-row groups
+  w.fused = off = align_up(off, 1024);
+  if (r < L.k * L.k && L.dtype == LBP_BF16 && L.k == 8 && r <= 16)
+    off += fused_scratch_bytes(L, r, nullptr);
   w.total = align_up(off, 256);
   return w;
 }
@@ -228,6 +243,21 @@ int lbp_backward(const void* x, const void* g_y, const void* W, void* g_x, void*
   if (r == L.k * L.k) return run_fullrank(x, g_y, W, g_x, g_W, L, wsb, st);
 
   uint32_t* status = reinterpret_cast<uint32_t*>(wsb);
+  if (fused_enabled() && fused_supported(L, plan)) {
+    // projection kernel, then one persistent kernel for both products with the
+    // expansion fused into the g_x_hat epilogue
+    if (int e = mark_phase(0, st)) return e;
+    auto after_projection = [](void*, cudaStream_t s) -> int {
+      if (int e = mark_phase(1, s)) return e;
+      return mark_phase(2, s);
+    };
+    if (int e = launch_fused(x, g_y, W, g_x, g_W, L, plan, wsb + lay.fused, status, st,
+                             after_projection, nullptr))
+      return e;
+    for (int ph = 3; ph <= 5; ++ph)
+      if (int e = mark_phase(ph, st)) return e;
+    return LBP_OK;
+  }
   void* x_hat = wsb + lay.x_hat;
   void* gy_hat = wsb + lay.gy_hat;
   float* gx_hat = reinterpret_cast<float*>(wsb + lay.gx_hat);

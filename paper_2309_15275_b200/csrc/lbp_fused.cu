@@ -1,0 +1,536 @@
+// Persistent kernel for the low-rank products and the expansion of Algorithm 1
+// (bf16 data, order k = 8, r <= 16), run after the projection kernel.
+//
+// One CTA per SM works through a static list of output tiles of the two
+// products, fp32 accumulators in TMEM, operands fed by TMA:
+//
+//   GW tile (i, j):  g_W[128 i .., BNw j ..] = g_y_hat^T x_hat      K = all low-rank rows
+//   GX tile (m, n):  g_x_hat[group m, BNx n ..] = g_y_hat[m] W      K = Cout
+//
+// A GX tile never leaves the chip as g_x_hat: the epilogue warps apply the
+// transposed bases (Eq. 7) to the accumulator and write g_x directly, while
+// the tensor core already works on the next tile (two accumulator slots in
+// TMEM, used alternately).
+//
+// Warp roles: warp 0 TMA producer, warp 1 TMEM owner and tcgen05 issuer,
+// warps 2-9 epilogue (two groups of four, alternating 32-column chunks of a
+// tile).  All roles walk the same tile list.  Every wait is bounded and an
+// expired wait is reported through the status block.
+#include <cuda_bf16.h>
+#include <cstdlib>
+
+#include "lbp_fused.cuh"
+#include "lbp_internal.h"
+#include "ptx_sm100.cuh"
+#include "wht_device.cuh"
+
+namespace lbp {
+namespace fused {
+
+constexpr int BM = 128, BK = 64;
+constexpr int kStages = 4;
+constexpr int kABytes = BM * BK * 2;             // 16 KB
+constexpr int kBBytes = 256 * BK * 2;            // 32 KB (up to 256 columns)
+constexpr int kStageBytes = kABytes + kBBytes;   // 48 KB
+constexpr int kChunkBytes = 64 * BK * 2;         // 8 KB: one 64-wide chunk of an MN-major tile
+constexpr int kEStride = 33;
+constexpr int kEBytes = BM * kEStride * 4;
+constexpr int kEGroups = 2;                      // epilogue groups of 4 warps (one per TMEM lane quarter)
+constexpr int kThreads = (2 + 4 * kEGroups) * 32;
+constexpr int kOffE = kStages * kStageBytes;
+constexpr int kOffBar = kOffE + kEGroups * kEBytes;
+constexpr int kSmemBytes = kOffBar + 256 + 1024;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kSlotCols = 256;   // two accumulator slots; tile number t of a CTA uses slot t & 1
+
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Optional role timeline (diagnostics): slot 0 kernel start, 2 producer done,
+// 3 MMA issuer done, 4 epilogue done, 5 first tile drained.
+__device__ __forceinline__ void trace_mark(const FusedParams& p, int slot, bool first_only = false) {
+  if (p.trace != nullptr) {
+    unsigned long long* t = p.trace + blockIdx.x * 8 + slot;
+    const unsigned long long now = global_ns();
+    if (first_only) {
+      if (*t == 0) *t = now;
+    } else {
+      atomicMax(t, now);
+    }
+  }
+}
+
+__device__ __forceinline__ int blocks_in_group(const FusedParams& p, int g) {
+  const int left = p.nb - g * p.bpt;
+  return left < p.bpt ? left : p.bpt;
+}
+
+// Tile list.  Tiles are numbered with the GW tiles (the larger ones) first and
+// dealt to the CTAs in a snake: round 0 forwards, round 1 backwards, ... so
+// that a CTA that got a large tile gets its next one last.
+struct Tile {
+  int is_gw;
+  int a, b;   // GW: (i, j) ; GX: (m, n)
+};
+__device__ __forceinline__ int tiles_of_cta(const FusedParams& p, int cta, int grid) {
+  const int total = p.n_gw_tiles + p.n_gx_tiles;
+  int n = 0;
+  for (int round = 0; round * grid < total; ++round) {
+    const int pos = (round & 1) ? (grid - 1 - cta) : cta;
+    if (round * grid + pos < total) ++n;
+  }
+  return n;
+}
+__device__ __forceinline__ Tile nth_tile(const FusedParams& p, int cta, int grid, int nth) {
+  const int total = p.n_gw_tiles + p.n_gx_tiles;
+  int seen = 0, id = 0;
+  for (int round = 0; round * grid < total; ++round) {
+    const int pos = (round & 1) ? (grid - 1 - cta) : cta;
+    const int t = round * grid + pos;
+    if (t < total) {
+      if (seen == nth) {
+        id = t;
+        break;
+      }
+      ++seen;
+    }
+  }
+  Tile tl;
+  if (id < p.n_gw_tiles) {
+    tl.is_gw = 1;
+    tl.a = id / p.nt_w;
+    tl.b = id - tl.a * p.nt_w;
+  } else {
+    id -= p.n_gw_tiles;
+    tl.is_gw = 0;
+    tl.a = id / p.n_tx;
+    tl.b = id - tl.a * p.n_tx;
+  }
+  return tl;
+}
+
+// ------------------------------------------------------------------ kernel ----
+template <int LB>
+__global__ void __launch_bounds__(kThreads, 1)
+    lbp_products_kernel(const __grid_constant__ CUtensorMap tm_gyhat_k,
+                        const __grid_constant__ CUtensorMap tm_gyhat_mn,
+                        const __grid_constant__ CUtensorMap tm_xhat,
+                        const __grid_constant__ CUtensorMap tm_w,
+                        const __grid_constant__ FusedParams p,
+                        const __grid_constant__ FusedBasis fb) {
+  constexpr int K = 8;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  float* E = reinterpret_cast<float*>(smem + kOffE);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kOffBar);
+  uint64_t* empty_bar = full_bar + kStages;
+  uint64_t* acc_full = empty_bar + kStages;   // [2]: accumulator slots
+  uint64_t* acc_empty = acc_full + 2;         // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int cta = blockIdx.x, grid = gridDim.x;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      ptx::mbar_init(&full_bar[s], 1);
+      ptx::mbar_init(&empty_bar[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      ptx::mbar_init(&acc_full[s], 1);
+      ptx::mbar_init(&acc_empty[s], 4 * kEGroups);
+    }
+    ptx::mbar_fence_init();
+    *abort_flag = 0;
+    ptx::prefetch_tensormap(&tm_gyhat_k);
+    ptx::prefetch_tensormap(&tm_gyhat_mn);
+    ptx::prefetch_tensormap(&tm_xhat);
+    ptx::prefetch_tensormap(&tm_w);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 0) trace_mark(p, 0);
+
+  const int my_tiles = tiles_of_cta(p, cta, grid);
+
+  if (warp == 0) {
+    // =========================== TMA producer ===========================
+    if (ptx::elect_one()) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int ti = 0; ti < my_tiles && ok; ++ti) {
+        const Tile tl = nth_tile(p, cta, grid, ti);
+        const int n_kb = tl.is_gw ? p.num_kb_w : p.num_kb_x;
+        const int bn = tl.is_gw ? p.BNw : p.BNx;
+        const uint32_t tx = static_cast<uint32_t>(kABytes + bn * BK * 2);
+        for (int kb = 0; kb < n_kb; ++kb) {
+          const int s = static_cast<int>(it % kStages);
+          if (!ptx::mbar_wait(&empty_bar[s], ((it / kStages) + 1) & 1u, p.status, (4u << 16) | 1u)) {
+            ok = false;
+            break;
+          }
+          uint8_t* sa = smem + s * kStageBytes;
+          uint8_t* sb = sa + kABytes;
+          ptx::mbar_expect_tx(&full_bar[s], tx);
+          if (tl.is_gw) {
+            // A = g_y_hat^T tile: stored (rows, Cout), MN-major, two 64-wide chunks
+            ptx::tma_load_2d(sa, &tm_gyhat_mn, &full_bar[s], tl.a * 128, kb * BK);
+            ptx::tma_load_2d(sa + kChunkBytes, &tm_gyhat_mn, &full_bar[s], tl.a * 128 + 64, kb * BK);
+            for (int c = 0; c < bn / 64; ++c)
+              ptx::tma_load_2d(sb + c * kChunkBytes, &tm_xhat, &full_bar[s], tl.b * bn + c * 64,
+                               kb * BK);
+          } else {
+            // A = g_y_hat rows of group m, K-major
+            ptx::tma_load_2d(sa, &tm_gyhat_k, &full_bar[s], kb * BK, tl.a * BM);
+            for (int c = 0; c < bn / 64; ++c)
+              ptx::tma_load_2d(sb + c * kChunkBytes, &tm_w, &full_bar[s], tl.b * bn + c * 64, kb * BK);
+          }
+          ++it;
+        }
+      }
+      if (!ok) *abort_flag = 1;
+      trace_mark(p, 2);
+    }
+  } else if (warp == 1) {
+    // =========================== tcgen05 issuer ===========================
+    if (ptx::elect_one()) {
+      uint32_t it = 0;
+      bool ok = true;
+      const uint32_t idesc_w = ptx::idesc_bf16(BM, p.BNw, true, true);
+      const uint32_t idesc_x = ptx::idesc_bf16(BM, p.BNx, false, true);
+      for (int ti = 0; ti < my_tiles && ok; ++ti) {
+        const Tile tl = nth_tile(p, cta, grid, ti);
+        const int slot = ti & 1;
+        const int n_kb = tl.is_gw ? p.num_kb_w : p.num_kb_x;
+        const uint32_t d_tmem = tmem_base + slot * kSlotCols;
+        const uint32_t idesc = tl.is_gw ? idesc_w : idesc_x;
+        const uint32_t uses = static_cast<uint32_t>(ti >> 1);   // earlier uses of this slot
+        // the accumulator slot must have been drained by the epilogue
+        if (!ptx::mbar_wait(&acc_empty[slot], (uses + 1) & 1u, p.status, (4u << 16) | 4u)) {
+          ok = false;
+          break;
+        }
+        for (int kb = 0; kb < n_kb; ++kb) {
+          const int s = static_cast<int>(it % kStages);
+          if (!ptx::mbar_wait(&full_bar[s], (it / kStages) & 1u, p.status, (4u << 16) | 3u)) {
+            ok = false;
+            break;
+          }
+          ptx::tc_fence_after_sync();
+          const uint32_t sa = ptx::smem_u32(smem + s * kStageBytes);
+          const uint32_t sb = sa + kABytes;
+#pragma unroll
+          for (int kk = 0; kk < BK / 16; ++kk) {
+            const uint64_t da = tl.is_gw ? ptx::smem_desc_sw128(sa + kk * 2048, kChunkBytes, 1024)
+                                         : ptx::smem_desc_sw128(sa + kk * 32, 16, 1024);
+            const uint64_t db = ptx::smem_desc_sw128(sb + kk * 2048, kChunkBytes, 1024);
+            ptx::mma_bf16_ss(d_tmem, da, db, idesc, (kb == 0 && kk == 0) ? 0u : 1u);
+          }
+          ptx::mma_commit(&empty_bar[s]);
+          ++it;
+        }
+        if (!ok) break;
+        ptx::mma_commit(&acc_full[slot]);
+      }
+      if (!ok) *abort_flag = 1;
+      trace_mark(p, 3);
+    }
+  } else {
+    // =========================== epilogue ===========================
+    const int eg = (warp - 2) >> 2;          // epilogue group: chunks eg, eg + kEGroups, ...
+    const int ew = (warp - 2) & 3;           // warp within the group
+    const int quarter = warp & 3;            // TMEM lane quarter this warp may read
+    const int etid = ew * 32 + lane;         // 0..127 within the group
+    const uint32_t lane_bits = static_cast<uint32_t>(quarter * 32) << 16;
+    float* const Eg = E + eg * (kEBytes / 4);
+    const int bar_id = 1 + eg;
+    for (int ti = 0; ti < my_tiles; ++ti) {
+      const Tile tl = nth_tile(p, cta, grid, ti);
+      const int slot = ti & 1;
+      const uint32_t uses = static_cast<uint32_t>(ti >> 1);
+      const uint32_t acc_col = slot * kSlotCols;
+      const bool ok = ptx::mbar_wait(&acc_full[slot], uses & 1u, p.status, (4u << 16) | 5u);
+      if (!__all_sync(0xffffffffu, ok)) *abort_flag = 1;
+      named_bar_sync(bar_id, 128);
+      if (*abort_flag) break;
+      ptx::tc_fence_after_sync();
+      if (etid == 0 && eg == 0) trace_mark(p, 5, true);
+      const int bn = tl.is_gw ? p.BNw : p.BNx;
+      bool released = false;
+
+      if (tl.is_gw) {
+        // ---- GW tile: g_W[128 i + row, BNw j + col] ----
+        const long long row = static_cast<long long>(tl.a) * 128 + quarter * 32 + lane;
+        for (int c0 = eg * 32; c0 < bn; c0 += 32 * kEGroups) {
+          uint32_t v[32];
+          ptx::tmem_ld_32x32(tmem_base + lane_bits + acc_col + c0, v);
+          ptx::tmem_ld_wait();
+          if (c0 + 32 * kEGroups >= bn) {
+            released = true;
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&acc_empty[slot]);
+          }
+          if (row < p.Cout) {
+            const long long colb = static_cast<long long>(tl.b) * bn + c0;
+            if (p.gw_bf16) {
+              __nv_bfloat16* d = static_cast<__nv_bfloat16*>(p.g_W) + row * p.Cin;
+#pragma unroll
+              for (int q = 0; q < 32; q += 8) {
+                if (colb + q < p.Cin) {
+                  uint4 o;
+                  o.x = pack_bf16x2(__uint_as_float(v[q]), __uint_as_float(v[q + 1]));
+                  o.y = pack_bf16x2(__uint_as_float(v[q + 2]), __uint_as_float(v[q + 3]));
+                  o.z = pack_bf16x2(__uint_as_float(v[q + 4]), __uint_as_float(v[q + 5]));
+                  o.w = pack_bf16x2(__uint_as_float(v[q + 6]), __uint_as_float(v[q + 7]));
+                  *reinterpret_cast<uint4*>(d + colb + q) = o;
+                }
+              }
+            } else {
+              float* d = static_cast<float*>(p.g_W) + row * p.Cin;
+#pragma unroll
+              for (int q = 0; q < 32; q += 4) {
+                if (colb + q < p.Cin)
+                  *reinterpret_cast<uint4*>(d + colb + q) = make_uint4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+              }
+            }
+          }
+        }
+      } else {
+        // ---- GX tile: expand g_x_hat (128 rows x BNx columns) into g_x ----
+        const int m = tl.a, n = tl.b;
+        const int bg = blocks_in_group(p, m);
+        constexpr int NCH = LB <= 4 ? 2 : 1;
+        constexpr int RUN = K / LB;
+        constexpr int CPT = 32 / NCH;       // threads across one 32-column chunk
+        constexpr int BSLOTS = 128 / CPT;   // blocks expanded concurrently
+        const int cc = etid % CPT, bs = etid / CPT;
+        for (int c0 = eg * 32; c0 < bn; c0 += 32 * kEGroups) {
+          uint32_t v[32];
+          ptx::tmem_ld_32x32(tmem_base + lane_bits + acc_col + c0, v);
+          ptx::tmem_ld_wait();
+          if (c0 + 32 * kEGroups >= bn) {
+            released = true;
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&acc_empty[slot]);
+          }
+          float* erow = Eg + (quarter * 32 + lane) * kEStride;
+#pragma unroll
+          for (int q = 0; q < 32; ++q) erow[q] = __uint_as_float(v[q]);
+          named_bar_sync(bar_id, 128);
+          const int ch = n * bn + c0 + cc * NCH;
+          if (ch < p.Cin) {
+            for (int bl = bs; bl < bg; bl += BSLOTS) {
+              float acc[LB][LB][NCH];
+              const float* eb = Eg + (bl * p.r) * kEStride + cc * NCH;
+#pragma unroll
+              for (int a = 0; a < LB; ++a) {
+#pragma unroll
+                for (int b = 0; b < LB; ++b) {
+                  const int q = fb.qmap[a * LB + b];
+#pragma unroll
+                  for (int c = 0; c < NCH; ++c) acc[a][b][c] = q >= 0 ? eb[q * kEStride + c] : 0.f;
+                }
+              }
+              hadamard_rows<LB, NCH>(acc);
+              hadamard_cols<LB, NCH>(acc);
+#pragma unroll
+              for (int a = 0; a < LB; ++a)
+#pragma unroll
+                for (int b = 0; b < LB; ++b)
+#pragma unroll
+                  for (int c = 0; c < NCH; ++c) acc[a][b][c] *= p.scale;
+              const int blk = m * p.bpt + bl;
+              const int bw = blk % p.Wb, t2 = blk / p.Wb, bh = t2 % p.Hb, b = t2 / p.Hb;
+              __nv_bfloat16* o = p.g_x +
+                                 ((static_cast<long long>(b) * p.H + bh * K) * p.W + bw * K) * p.Cin + ch;
+#pragma unroll
+              for (int u = 0; u < K; ++u) {
+#pragma unroll
+                for (int vv = 0; vv < K; ++vv) {
+                  __nv_bfloat16* dst = o + (static_cast<long long>(u) * p.W + vv) * p.Cin;
+                  if constexpr (NCH == 2) {
+                    *reinterpret_cast<uint32_t*>(dst) =
+                        pack_bf16x2(acc[u / RUN][vv / RUN][0], acc[u / RUN][vv / RUN][1]);
+                  } else {
+                    *dst = __float2bfloat16_rn(acc[u / RUN][vv / RUN][0]);
+                  }
+                }
+              }
+            }
+          }
+          named_bar_sync(bar_id, 128);
+        }
+      }
+      if (!released) {   // this group had no chunk of the tile
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&acc_empty[slot]);
+      }
+    }
+    if (etid == 0) trace_mark(p, 4);   // latest of the groups
+  }
+
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace fused
+
+// --------------------------------------------------------------- launcher ----
+bool fused_supported(const lbp_layer& L, const BasisPlan& bp) {
+  return L.dtype == LBP_BF16 && L.k == 8 && bp.r <= 16 && bp.LB <= 8;
+}
+
+size_t fused_scratch_bytes(const lbp_layer& L, int r, FusedLayout* lay) {
+  const long long nb = static_cast<long long>(L.B) * (L.H / L.k) * (L.W / L.k);
+  const int bpt = 128 / r;
+  const long long G = (nb + bpt - 1) / bpt;
+  FusedLayout l;
+  size_t off = 0;
+  l.x_hat = off;
+  off += static_cast<size_t>(G) * 128 * L.Cin * 2;
+  off = (off + 1023) / 1024 * 1024;
+  l.gy_hat = off;
+  off += static_cast<size_t>(G) * 128 * L.Cout * 2;
+  off = (off + 1023) / 1024 * 1024;
+  l.trace = off;
+  off += kFusedTraceBytes;
+  l.total = (off + 1023) / 1024 * 1024;
+  l.G = static_cast<int>(G);
+  l.bpt = bpt;
+  if (lay) *lay = l;
+  return l.total;
+}
+
+int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void* g_W,
+                 const lbp_layer& L, const BasisPlan& bp, uint8_t* scratch, uint32_t* status,
+                 cudaStream_t stream, FusedPhaseHook hook, void* hook_arg) {
+  using namespace fused;
+  FusedLayout lay;
+  fused_scratch_bytes(L, bp.r, &lay);
+  const int K = L.k;
+  int dev = 0, sms = 0;
+  LBP_CUDA_TRY(cudaGetDevice(&dev));
+  LBP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  FusedParams p{};
+  p.Hb = L.H / K;
+  p.Wb = L.W / K;
+  p.nb = L.B * p.Hb * p.Wb;
+  p.H = L.H;
+  p.W = L.W;
+  p.r = bp.r;
+  p.bpt = lay.bpt;
+  p.G = lay.G;
+  p.Cin = L.Cin;
+  p.Cout = L.Cout;
+  // Column tiles are multiples of 64 (one TMA chunk) up to 256.  Each
+  // candidate pair is scored by the operand bytes of the busiest CTA under the
+  // snake assignment of the tile list (the kernel is bound by operand traffic).
+  p.num_kb_x = (L.Cout + BK - 1) / BK;
+  p.mt_w = (L.Cout + 127) / 128;
+  p.num_kb_w = p.G * (BM / BK);
+  const int cin64 = (L.Cin + 63) / 64 * 64;
+  double best = -1.0;
+  for (int bnw = 64; bnw <= 256; bnw += 64) {
+    for (int bnx = 64; bnx <= 256; bnx += 64) {
+      if (bnw > cin64 || bnx > cin64) continue;
+      const int nt_w = (L.Cin + bnw - 1) / bnw, n_tx = (L.Cin + bnx - 1) / bnx;
+      const int n_gw = p.mt_w * nt_w, n_gx = p.G * n_tx;
+      const double gw_cost = static_cast<double>(p.num_kb_w) * (kABytes + bnw * 128.0);
+      const double gx_cost = static_cast<double>(p.num_kb_x) * (kABytes + bnx * 128.0) +
+                             6000.0 * bnx;   // plus the expansion of the tile
+      const int total = n_gw + n_gx;
+      const int grid = total < sms ? total : sms;
+      double worst = 0.0;
+      for (int c = 0; c < grid; ++c) {
+        double load = 0.0;
+        for (int round = 0; round * grid < total; ++round) {
+          const int t = round * grid + ((round & 1) ? grid - 1 - c : c);
+          if (t < total) load += t < n_gw ? gw_cost : gx_cost;
+        }
+        if (load > worst) worst = load;
+      }
+      if (best < 0 || worst < best) {
+        best = worst;
+        p.BNw = bnw;
+        p.BNx = bnx;
+      }
+    }
+  }
+  p.n_tx = (L.Cin + p.BNx - 1) / p.BNx;
+  p.nt_w = (L.Cin + p.BNw - 1) / p.BNw;
+  p.n_gx_tiles = p.G * p.n_tx;
+  p.n_gw_tiles = p.mt_w * p.nt_w;
+  p.gw_bf16 = L.gw_dtype == LBP_BF16 ? 1 : 0;
+  p.scale = 1.0f / static_cast<float>(K);
+  p.x_hat = reinterpret_cast<__nv_bfloat16*>(scratch + lay.x_hat);
+  p.gy_hat = reinterpret_cast<__nv_bfloat16*>(scratch + lay.gy_hat);
+  p.g_x = static_cast<__nv_bfloat16*>(g_x);
+  p.g_W = g_W;
+  p.status = status;
+  p.trace = nullptr;
+  if (const char* e = std::getenv("LBP_FUSED_TRACE")) {
+    if (e[0] == '1') {
+      p.trace = reinterpret_cast<unsigned long long*>(scratch + lay.trace);
+      LBP_CUDA_TRY(cudaMemsetAsync(p.trace, 0, kFusedTraceBytes, stream));
+    }
+  }
+
+  FusedBasis fb;
+  for (int n = 0; n < 64; ++n) fb.qmap[n] = -1;
+  for (int a = 0; a < bp.LB; ++a)
+    for (int b = 0; b < bp.LB; ++b) fb.qmap[a * bp.LB + b] = bp.qmap[a * bp.LB + b];
+
+  // Algorithm 1, steps 1-2: x_hat and g_y_hat, rows padded to 128-row groups
+  if (int e = launch_project2(g_y, p.gy_hat, L.Cout, x, p.x_hat, L.Cin, LBP_BF16, L.B, L.H, L.W, bp,
+                              RowMap{p.bpt, BM}, status, stream))
+    return e;
+  if (hook != nullptr)
+    if (int e = hook(hook_arg, stream)) return e;
+
+  CUtensorMap tm_gyhat_k, tm_gyhat_mn, tm_xhat, tm_w;
+  const long long rows = static_cast<long long>(p.G) * BM;
+  if (int e = encode_matrix_tensor_map(&tm_gyhat_k, p.gy_hat, rows, L.Cout, BM)) return e;
+  if (int e = encode_matrix_tensor_map(&tm_gyhat_mn, p.gy_hat, rows, L.Cout, BK)) return e;
+  if (int e = encode_matrix_tensor_map(&tm_xhat, p.x_hat, rows, L.Cin, BK)) return e;
+  if (int e = encode_matrix_tensor_map(&tm_w, W, L.Cout, L.Cin, BK)) return e;
+
+  const int total_tiles = p.n_gw_tiles + p.n_gx_tiles;
+  const int grid = total_tiles < sms ? total_tiles : sms;
+
+  auto launch = [&](auto kern) -> int {
+    LBP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    kern<<<grid, kThreads, kSmemBytes, stream>>>(tm_gyhat_k, tm_gyhat_mn, tm_xhat, tm_w, p, fb);
+    count_launch();
+    LBP_CUDA_TRY(cudaGetLastError());
+    return LBP_OK;
+  };
+  switch (bp.LB) {
+    case 1: return launch(lbp_products_kernel<1>);
+    case 2: return launch(lbp_products_kernel<2>);
+    case 4: return launch(lbp_products_kernel<4>);
+    case 8: return launch(lbp_products_kernel<8>);
+  }
+  return LBP_ERR_BASIS;
+}
+
+}  // namespace lbp

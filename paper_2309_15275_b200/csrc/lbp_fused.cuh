@@ -1,0 +1,52 @@
+// Declarations of the persistent products + expansion kernel (bf16, k = 8, r <= 16).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "lbp_internal.h"
+
+namespace lbp {
+
+struct FusedParams {
+  // token grid and low-rank row layout: block blk of group g = blk / bpt owns rows
+  // g * 128 + (blk % bpt) * r ... + r - 1 of x_hat / g_y_hat; the other rows of a
+  // group are zero
+  int32_t nb, Hb, Wb, H, W, r, bpt, G;
+  int32_t Cin, Cout;
+  // products
+  int32_t BNx, n_tx, num_kb_x;            // GX: column tile, tiles per row group, k-blocks (Cout / 64)
+  int32_t BNw, mt_w, nt_w, num_kb_w;      // GW: 128 x BNw tiles, k-blocks (G * 2)
+  int32_t n_gx_tiles, n_gw_tiles;
+  int32_t gw_bf16;
+  float scale;                            // 1/k
+  __nv_bfloat16* x_hat;
+  __nv_bfloat16* gy_hat;
+  __nv_bfloat16* g_x;
+  void* g_W;
+  uint32_t* status;
+  unsigned long long* trace;              // optional role timeline, 8 slots per CTA (null = off)
+};
+
+struct FusedBasis {
+  int16_t qmap[64];   // natural-order LB x LB position -> basis slot, -1 unused
+};
+
+constexpr size_t kFusedTraceBytes = 256 * 8 * 8;   // last bytes of the scratch region
+
+struct FusedLayout {
+  size_t x_hat, gy_hat, trace, total;
+  int G, bpt;
+};
+
+// Called between the projection launch and the products launch (phase events).
+using FusedPhaseHook = int (*)(void* arg, cudaStream_t stream);
+
+bool fused_supported(const lbp_layer& L, const BasisPlan& bp);
+size_t fused_scratch_bytes(const lbp_layer& L, int r, FusedLayout* lay);
+int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void* g_W,
+                 const lbp_layer& L, const BasisPlan& bp, uint8_t* scratch, uint32_t* status,
+                 cudaStream_t stream, FusedPhaseHook hook, void* hook_arg);
+
+}  // namespace lbp
