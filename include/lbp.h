@@ -149,6 +149,34 @@ int lbp_backward_fullrank(const void* x, const void* g_y, const void* W,
                           void* g_x, void* g_W, const lbp_layer* layer,
                           void* ws, size_t ws_bytes, void* stream);
 
+/* No counterpart in the paper: a packaging variant of lbp_backward for callers
+ * that cannot allocate device memory.  Examples are a server that handed all
+ * device memory to its own pool at start-up and forbids cudaMalloc afterwards,
+ * a plug-in whose host framework passes it nothing but input and output
+ * buffers, and code on a path where an allocation would synchronise the device
+ * or is not permitted.  The scratch that lbp_backward takes from the caller
+ * comes here from an array of LBP_STATIC_SCRATCH_BYTES that is part of the
+ * library image: every GPU on which the library is loaded holds that much
+ * memory until the process exits.
+ *  - Same arguments, layouts and results as lbp_backward, minus ws / ws_bytes.
+ *    The call allocates and frees nothing.
+ *  - Layers with lbp_workspace_bytes(layer, r) > LBP_STATIC_SCRATCH_BYTES are
+ *    rejected with LBP_ERR_WORKSPACE before anything is enqueued.
+ *  - The first call on a device looks up the array's device address (no
+ *    allocation, but a runtime query): make that first call outside any stream
+ *    capture.  The device that is current at the call owns the scratch used.
+ *  - All calls on a device share the one array.  Its status block is cleared
+ *    on `stream` at the start of every call; everything else in it is
+ *    overwritten before it is read.  Two calls whose device work overlaps in
+ *    time (different streams, or different host threads) race on the array:
+ *    order them on one stream or with events.
+ *  - The status block is not reachable through lbp_poll_status; a caller that
+ *    needs the device status uses lbp_backward with its own workspace. */
+#define LBP_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+int lbp_backward_static(const void* x, const void* g_y, const void* W,
+                        void* g_x, void* g_W, const lbp_layer* layer,
+                        const lbp_basis* set, int r, void* stream);
+
 /* Synchronises `stream`, reads the device status word at the start of ws and
  * clears it.  Returns LBP_OK, LBP_ERR_TIMEOUT (a bounded wait in a kernel
  * expired; outputs of that call are undefined, the context stays usable) or

@@ -8,5 +8,5 @@ from .binding import (  # noqa: F401
     alloc_workspace, lbp_backward, lbp_backward_fullrank, lbp_basis_matrix, lbp_expand,
     lbp_flops, lbp_poll_status, lbp_project, lbp_select_bases, lbp_status_bytes,
     lbp_status_string, lbp_workspace_bytes, lbp_launch_count, lbp_phase_count, lbp_phase_name,
-    lbp_set_phase_events,
+    lbp_set_phase_events, lbp_backward_static, STATIC_SCRATCH_BYTES,
 )

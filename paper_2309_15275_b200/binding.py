@@ -77,6 +77,9 @@ def _lib() -> C.CDLL:
         lib.lbp_backward_fullrank.restype = i32
         lib.lbp_poll_status.argtypes = [vp, vp]
         lib.lbp_poll_status.restype = i32
+        lib.lbp_backward_static.argtypes = [vp, vp, vp, vp, vp, C.POINTER(Layer), C.POINTER(Basis),
+                                            i32, vp]
+        lib.lbp_backward_static.restype = i32
         lib.lbp_launch_count.argtypes = []
         lib.lbp_launch_count.restype = C.c_longlong
         lib.lbp_set_phase_events.argtypes = [C.POINTER(vp), i32]
@@ -92,7 +95,7 @@ def _lib() -> C.CDLL:
 EXPORTED = ("lbp_select_bases", "lbp_basis_matrix", "lbp_flops", "lbp_status_string",
             "lbp_last_cuda_error", "lbp_workspace_bytes", "lbp_status_bytes", "lbp_project",
             "lbp_expand", "lbp_backward", "lbp_backward_fullrank", "lbp_poll_status",
-            "lbp_launch_count", "lbp_set_phase_events", "lbp_phase_count", "lbp_phase_name")
+            "lbp_backward_static", "lbp_launch_count", "lbp_set_phase_events", "lbp_phase_count", "lbp_phase_name")
 
 
 def _check(status: int, where: str) -> None:
@@ -245,6 +248,24 @@ def lbp_backward_fullrank(x, g_y, W, k: int, *, gw_dtype: torch.dtype = torch.fl
                                         _dev(g_x, "g_x"), _dev(g_W, "g_W"), C.byref(lay),
                                         _dev(ws, "ws"), ws.numel(), _stream()),
            "lbp_backward_fullrank")
+    return g_x, g_W
+
+
+STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
+
+
+def lbp_backward_static(x, g_y, W, k: int, bases, *, g_x, g_W):
+    """lbp_backward on the scratch array built into the library: no workspace
+    argument and no allocation inside the call.  The caller passes the output
+    tensors g_x (B,H,W,Cin) and g_W (Cout,Cin); layers whose scratch need exceeds
+    STATIC_SCRATCH_BYTES raise LbpError (status 7)."""
+    B, H, Wd, Cin = x.shape
+    Cout = g_y.shape[-1]
+    lay = _layer(B, H, Wd, Cin, Cout, k, _dtype_code(x.dtype), _dtype_code(g_W.dtype))
+    _check(_lib().lbp_backward_static(_dev(x, "x"), _dev(g_y, "g_y"), _dev(W, "W"),
+                                      _dev(g_x, "g_x"), _dev(g_W, "g_W"), C.byref(lay),
+                                      _bases(bases), len(bases), _stream()),
+           "lbp_backward_static")
     return g_x, g_W
 
 
