@@ -292,12 +292,13 @@ _PHASE_KEEPALIVE = None
 
 def lbp_set_phase_events(events) -> None:
     """events: list of torch.cuda.Event (already created with enable_timing=True
-    and recorded once so their handles exist), or None to switch the hook off."""
+    and recorded once so their handles exist; an entry may be None to skip that
+    phase boundary), or None to switch the hook off."""
     global _PHASE_KEEPALIVE
     if events is None:
         _check(_lib().lbp_set_phase_events(None, 0), "lbp_set_phase_events")
         _PHASE_KEEPALIVE = None
         return
-    arr = (C.c_void_p * len(events))(*[e.cuda_event for e in events])
+    arr = (C.c_void_p * len(events))(*[None if e is None else e.cuda_event for e in events])
     _check(_lib().lbp_set_phase_events(arr, len(events)), "lbp_set_phase_events")
     _PHASE_KEEPALIVE = (arr, list(events))
