@@ -33,7 +33,7 @@ constexpr int kABytes = BM * BK * 2;             // 16 KB
 constexpr int kBBytes = 256 * BK * 2;            // 32 KB (up to 256 columns)
 constexpr int kStageBytes = kABytes + kBBytes;   // 48 KB
 constexpr int kChunkBytes = 64 * BK * 2;         // 8 KB: one 64-wide chunk of an MN-major tile
-constexpr int kEStride = 33;
+constexpr int kEStride = 32;   // fp32 words per staged row; 16-byte chunk c of row i sits at chunk c ^ (i & 7)
 constexpr int kEBytes = BM * kEStride * 4;
 constexpr int kEGroups = 2;                      // epilogue groups of 4 warps (one per TMEM lane quarter)
 constexpr int kThreads = (2 + 4 * kEGroups) * 32;
@@ -313,11 +313,13 @@ __global__ void __launch_bounds__(kThreads, 1)
         // ---- GX tile: expand g_x_hat (128 rows x BNx columns) into g_x ----
         const int m = tl.a, n = tl.b;
         const int bg = blocks_in_group(p, m);
-        constexpr int NCH = LB <= 4 ? 2 : 1;
+        constexpr int NCH = LB <= 4 ? 4 : 1;   // channels per thread
         constexpr int RUN = K / LB;
         constexpr int CPT = 32 / NCH;       // threads across one 32-column chunk
         constexpr int BSLOTS = 128 / CPT;   // blocks expanded concurrently
         const int cc = etid % CPT, bs = etid / CPT;
+        // element offsets of a token inside a block fit 32 bits (checked on the host)
+        const int tok_stride = p.Cin, row_stride = p.W * p.Cin;
         for (int c0 = eg * 32; c0 < bn; c0 += 32 * kEGroups) {
           uint32_t v[32];
           ptx::tmem_ld_32x32(tmem_base + lane_bits + acc_col + c0, v);
@@ -328,46 +330,66 @@ __global__ void __launch_bounds__(kThreads, 1)
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&acc_empty[slot]);
           }
-          float* erow = Eg + (quarter * 32 + lane) * kEStride;
+          const int erow_i = quarter * 32 + lane;
+          uint4* erow = reinterpret_cast<uint4*>(Eg + erow_i * kEStride);
 #pragma unroll
-          for (int q = 0; q < 32; ++q) erow[q] = __uint_as_float(v[q]);
+          for (int q = 0; q < 8; ++q)
+            erow[q ^ (erow_i & 7)] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
           named_bar_sync(bar_id, 128);
           const int ch = n * bn + c0 + cc * NCH;
           if (ch < p.Cin) {
             for (int bl = bs; bl < bg; bl += BSLOTS) {
               float acc[LB][LB][NCH];
-              const float* eb = Eg + (bl * p.r) * kEStride + cc * NCH;
+              const int row_b = bl * p.r;
 #pragma unroll
               for (int a = 0; a < LB; ++a) {
 #pragma unroll
                 for (int b = 0; b < LB; ++b) {
                   const int q = fb.qmap[a * LB + b];
-#pragma unroll
-                  for (int c = 0; c < NCH; ++c) acc[a][b][c] = q >= 0 ? eb[q * kEStride + c] : 0.f;
+                  const int row_q = row_b + q;
+                  if constexpr (NCH == 4) {
+                    float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (q >= 0)
+                      f = *reinterpret_cast<const float4*>(Eg + row_q * kEStride + ((cc ^ (row_q & 7)) << 2));
+                    acc[a][b][0] = f.x;
+                    acc[a][b][1] = f.y;
+                    acc[a][b][2] = f.z;
+                    acc[a][b][3] = f.w;
+                  } else {
+                    acc[a][b][0] =
+                        q >= 0 ? Eg[row_q * kEStride + (((cc >> 2) ^ (row_q & 7)) << 2) + (cc & 3)] : 0.f;
+                  }
                 }
               }
               hadamard_rows<LB, NCH>(acc);
               hadamard_cols<LB, NCH>(acc);
-#pragma unroll
-              for (int a = 0; a < LB; ++a)
-#pragma unroll
-                for (int b = 0; b < LB; ++b)
-#pragma unroll
-                  for (int c = 0; c < NCH; ++c) acc[a][b][c] *= p.scale;
               const int blk = m * p.bpt + bl;
               const int bw = blk % p.Wb, t2 = blk / p.Wb, bh = t2 % p.Hb, b = t2 / p.Hb;
               __nv_bfloat16* o = p.g_x +
                                  ((static_cast<long long>(b) * p.H + bh * K) * p.W + bw * K) * p.Cin + ch;
+              // each of the LB x LB values covers a RUN x RUN patch of tokens: scale,
+              // round and pack once, store RUN * RUN times
 #pragma unroll
-              for (int u = 0; u < K; ++u) {
+              for (int a = 0; a < LB; ++a) {
 #pragma unroll
-                for (int vv = 0; vv < K; ++vv) {
-                  __nv_bfloat16* dst = o + (static_cast<long long>(u) * p.W + vv) * p.Cin;
-                  if constexpr (NCH == 2) {
-                    *reinterpret_cast<uint32_t*>(dst) =
-                        pack_bf16x2(acc[u / RUN][vv / RUN][0], acc[u / RUN][vv / RUN][1]);
+                for (int b2 = 0; b2 < LB; ++b2) {
+                  if constexpr (NCH == 4) {
+                    uint2 pk;
+                    pk.x = pack_bf16x2(acc[a][b2][0] * p.scale, acc[a][b2][1] * p.scale);
+                    pk.y = pack_bf16x2(acc[a][b2][2] * p.scale, acc[a][b2][3] * p.scale);
+#pragma unroll
+                    for (int du = 0; du < RUN; ++du)
+#pragma unroll
+                      for (int dv = 0; dv < RUN; ++dv)
+                        *reinterpret_cast<uint2*>(o + (a * RUN + du) * row_stride +
+                                                  (b2 * RUN + dv) * tok_stride) = pk;
                   } else {
-                    *dst = __float2bfloat16_rn(acc[u / RUN][vv / RUN][0]);
+                    const __nv_bfloat16 hv = __float2bfloat16_rn(acc[a][b2][0] * p.scale);
+#pragma unroll
+                    for (int du = 0; du < RUN; ++du)
+#pragma unroll
+                      for (int dv = 0; dv < RUN; ++dv)
+                        o[(a * RUN + du) * row_stride + (b2 * RUN + dv) * tok_stride] = hv;
                   }
                 }
               }
@@ -397,7 +419,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 
 // --------------------------------------------------------------- launcher ----
 bool fused_supported(const lbp_layer& L, const BasisPlan& bp) {
-  return L.dtype == LBP_BF16 && L.k == 8 && bp.r <= 16 && bp.LB <= 8;
+  // the epilogue addresses the tokens of a block with 32-bit element offsets
+  const long long block_span = 8ll * L.W * L.Cin;
+  return L.dtype == LBP_BF16 && L.k == 8 && bp.r <= 16 && bp.LB <= 8 && block_span < (1ll << 31);
 }
 
 size_t fused_scratch_bytes(const lbp_layer& L, int r, FusedLayout* lay) {
