@@ -169,6 +169,10 @@ __global__ void __launch_bounds__(kThreads, 1)
   if (warp == 0) {
     // =========================== TMA producer ===========================
     if (ptx::elect_one()) {
+      // The kernel is launched with programmatic stream serialization: everything
+      // above overlaps the tail of the projection kernel; its results (x_hat,
+      // g_y_hat) may only be read after this wait.
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       uint32_t it = 0;
       bool ok = true;
       for (int ti = 0; ti < my_tiles && ok; ++ti) {
@@ -543,7 +547,17 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
 
   auto launch = [&](auto kern) -> int {
     LBP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    kern<<<grid, kThreads, kSmemBytes, stream>>>(tm_gyhat_k, tm_gyhat_mn, tm_xhat, tm_w, p, fb);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    LBP_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tm_gyhat_k, tm_gyhat_mn, tm_xhat, tm_w, p, fb));
     count_launch();
     LBP_CUDA_TRY(cudaGetLastError());
     return LBP_OK;

@@ -93,6 +93,9 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
     ptx::prefetch_tensormap(&tmap0);
     ptx::prefetch_tensormap(&tmap1);
   }
+  // a kernel launched behind this one with programmatic serialization may set
+  // itself up as SMs free up; it still waits for this grid before reading
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   __syncthreads();
 
   const uint32_t first = blockIdx.x * NW + warp;
