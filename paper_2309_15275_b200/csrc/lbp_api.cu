@@ -146,10 +146,10 @@ static Layout plan_layout(const lbp_layer& L, int r) {
   }
   w.splitk = off = align_up(off, 1024);
   off += w.splitk_bytes;
-  // scratch of the persistent products kernel (bf16, k = 8, r <= 16): x_hat and
+  // scratch of the persistent products kernel (bf16, r <= 16): x_hat and
   // g_y_hat with rows padded to 128-row groups
   w.fused = off = align_up(off, 1024);
-  if (r < L.k * L.k && L.dtype == LBP_BF16 && L.k == 8 && r <= 16)
+  if (r < L.k * L.k && L.dtype == LBP_BF16 && r <= 16)
     off += fused_scratch_bytes(L, r, nullptr);
   w.total = align_up(off, 256);
   return w;

@@ -1,5 +1,5 @@
 // Persistent kernel for the low-rank products and the expansion of Algorithm 1
-// (bf16 data, order k = 8, r <= 16), run after the projection kernel.
+// (bf16 data, r <= 16), run after the projection kernel.
 //
 // One CTA per SM works through a static list of output tiles of the two
 // products, fp32 accumulators in TMEM, operands fed by TMA:
@@ -115,7 +115,7 @@ __device__ __forceinline__ Tile nth_tile(const FusedParams& p, int cta, int grid
 }
 
 // ------------------------------------------------------------------ kernel ----
-template <int LB>
+template <int K, int LB>
 __global__ void __launch_bounds__(kThreads, 1)
     lbp_products_kernel(const __grid_constant__ CUtensorMap tm_gyhat_k,
                         const __grid_constant__ CUtensorMap tm_gyhat_mn,
@@ -123,7 +123,6 @@ __global__ void __launch_bounds__(kThreads, 1)
                         const __grid_constant__ CUtensorMap tm_w,
                         const __grid_constant__ FusedParams p,
                         const __grid_constant__ FusedBasis fb) {
-  constexpr int K = 8;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -317,7 +316,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         // ---- GX tile: expand g_x_hat (128 rows x BNx columns) into g_x ----
         const int m = tl.a, n = tl.b;
         const int bg = blocks_in_group(p, m);
-        constexpr int NCH = LB <= 4 ? 4 : 1;   // channels per thread
+        // channels per thread (the 8 x 8 array of order 8 leaves registers for one)
+        constexpr int NCH = LB <= 4 ? 4 : (K >= 16 ? 2 : 1);
         constexpr int RUN = K / LB;
         constexpr int CPT = 32 / NCH;       // threads across one 32-column chunk
         constexpr int BSLOTS = 128 / CPT;   // blocks expanded concurrently
@@ -359,6 +359,13 @@ __global__ void __launch_bounds__(kThreads, 1)
                     acc[a][b][1] = f.y;
                     acc[a][b][2] = f.z;
                     acc[a][b][3] = f.w;
+                  } else if constexpr (NCH == 2) {
+                    float2 f = make_float2(0.f, 0.f);
+                    if (q >= 0)
+                      f = *reinterpret_cast<const float2*>(Eg + row_q * kEStride +
+                                                           (((cc >> 1) ^ (row_q & 7)) << 2) + (cc & 1) * 2);
+                    acc[a][b][0] = f.x;
+                    acc[a][b][1] = f.y;
                   } else {
                     acc[a][b][0] =
                         q >= 0 ? Eg[row_q * kEStride + (((cc >> 2) ^ (row_q & 7)) << 2) + (cc & 3)] : 0.f;
@@ -387,13 +394,21 @@ __global__ void __launch_bounds__(kThreads, 1)
                       for (int dv = 0; dv < RUN; ++dv)
                         *reinterpret_cast<uint2*>(o + (a * RUN + du) * row_stride +
                                                   (b2 * RUN + dv) * tok_stride) = pk;
-                  } else {
+                  } else if constexpr (NCH == 1) {
                     const __nv_bfloat16 hv = __float2bfloat16_rn(acc[a][b2][0] * p.scale);
 #pragma unroll
                     for (int du = 0; du < RUN; ++du)
 #pragma unroll
                       for (int dv = 0; dv < RUN; ++dv)
                         o[(a * RUN + du) * row_stride + (b2 * RUN + dv) * tok_stride] = hv;
+                  } else {
+                    const uint32_t pk = pack_bf16x2(acc[a][b2][0] * p.scale, acc[a][b2][1] * p.scale);
+#pragma unroll
+                    for (int du = 0; du < RUN; ++du)
+#pragma unroll
+                      for (int dv = 0; dv < RUN; ++dv)
+                        *reinterpret_cast<uint32_t*>(o + (a * RUN + du) * row_stride +
+                                                     (b2 * RUN + dv) * tok_stride) = pk;
                   }
                 }
               }
@@ -424,8 +439,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 // --------------------------------------------------------------- launcher ----
 bool fused_supported(const lbp_layer& L, const BasisPlan& bp) {
   // the epilogue addresses the tokens of a block with 32-bit element offsets
-  const long long block_span = 8ll * L.W * L.Cin;
-  return L.dtype == LBP_BF16 && L.k == 8 && bp.r <= 16 && bp.LB <= 8 && block_span < (1ll << 31);
+  const long long block_span = static_cast<long long>(L.k) * L.W * L.Cin;
+  return L.dtype == LBP_BF16 && (L.k == 4 || L.k == 8 || L.k == 16) && bp.r <= 16 && bp.LB <= 8 &&
+         bp.LB <= L.k && block_span < (1ll << 31);
 }
 
 size_t fused_scratch_bytes(const lbp_layer& L, int r, FusedLayout* lay) {
@@ -562,11 +578,18 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
     LBP_CUDA_TRY(cudaGetLastError());
     return LBP_OK;
   };
-  switch (bp.LB) {
-    case 1: return launch(lbp_products_kernel<1>);
-    case 2: return launch(lbp_products_kernel<2>);
-    case 4: return launch(lbp_products_kernel<4>);
-    case 8: return launch(lbp_products_kernel<8>);
+  switch (K * 100 + bp.LB) {
+    case 401: return launch(lbp_products_kernel<4, 1>);
+    case 402: return launch(lbp_products_kernel<4, 2>);
+    case 404: return launch(lbp_products_kernel<4, 4>);
+    case 801: return launch(lbp_products_kernel<8, 1>);
+    case 802: return launch(lbp_products_kernel<8, 2>);
+    case 804: return launch(lbp_products_kernel<8, 4>);
+    case 808: return launch(lbp_products_kernel<8, 8>);
+    case 1601: return launch(lbp_products_kernel<16, 1>);
+    case 1602: return launch(lbp_products_kernel<16, 2>);
+    case 1604: return launch(lbp_products_kernel<16, 4>);
+    case 1608: return launch(lbp_products_kernel<16, 8>);
   }
   return LBP_ERR_BASIS;
 }

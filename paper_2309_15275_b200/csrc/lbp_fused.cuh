@@ -1,4 +1,4 @@
-// Declarations of the persistent products + expansion kernel (bf16, k = 8, r <= 16).
+// Declarations of the persistent products + expansion kernel (bf16, r <= 16).
 #pragma once
 
 #include <cuda.h>
