@@ -285,6 +285,16 @@ Tiling choose_tiling(long long M, long long N, long long K, int sms) {
 int launch_gemm_fp32(const float* A, bool a_mn_major, const float* Bm, float* D, long long M,
                      long long N, long long K, cudaStream_t stream);
 
+int launch_splitk_reduce(const float* planes, void* D, long long mn, int splits, bool d_bf16,
+                         cudaStream_t stream) {
+  const long long threads = (mn + 3) / 4;
+  splitk_reduce_kernel<<<static_cast<unsigned>((threads + 255) / 256), 256, 0, stream>>>(
+      planes, D, mn, splits, d_bf16 ? 1 : 0);
+  count_launch();
+  LBP_CUDA_TRY(cudaGetLastError());
+  return LBP_OK;
+}
+
 size_t gemm_splitk_ws_bytes(long long M, long long N, long long K, int in_dtype) {
   if (in_dtype != LBP_BF16) return 0;
   // Enough for the most split tiling the planner can pick on a device with up

@@ -17,6 +17,7 @@
 // tile).  All roles walk the same tile list.  Every wait is bounded and an
 // expired wait is reported through the status block.
 #include <cuda_bf16.h>
+#include <cstdio>
 #include <cstdlib>
 
 #include "lbp_fused.cuh"
@@ -75,7 +76,9 @@ __device__ __forceinline__ int blocks_in_group(const FusedParams& p, int g) {
 // that a CTA that got a large tile gets its next one last.
 struct Tile {
   int is_gw;
-  int a, b;   // GW: (i, j) ; GX: (m, n)
+  int a, b;          // GW: (i, j) ; GX: (m, n)
+  int kb0, n_kb;     // k-block range of the tile (a K slice for GW)
+  int slice;
 };
 __device__ __forceinline__ int tiles_of_cta(const FusedParams& p, int cta, int grid) {
   const int total = p.n_gw_tiles + p.n_gx_tiles;
@@ -103,13 +106,21 @@ __device__ __forceinline__ Tile nth_tile(const FusedParams& p, int cta, int grid
   Tile tl;
   if (id < p.n_gw_tiles) {
     tl.is_gw = 1;
-    tl.a = id / p.nt_w;
-    tl.b = id - tl.a * p.nt_w;
+    const int t = id / p.gw_splits;
+    tl.slice = id - t * p.gw_splits;
+    tl.a = t / p.nt_w;
+    tl.b = t - tl.a * p.nt_w;
+    tl.kb0 = tl.slice * p.kb_per_split_w;
+    const int end = tl.kb0 + p.kb_per_split_w;
+    tl.n_kb = (end < p.num_kb_w ? end : p.num_kb_w) - tl.kb0;
   } else {
     id -= p.n_gw_tiles;
     tl.is_gw = 0;
+    tl.slice = 0;
     tl.a = id / p.n_tx;
     tl.b = id - tl.a * p.n_tx;
+    tl.kb0 = 0;
+    tl.n_kb = p.num_kb_x;
   }
   return tl;
 }
@@ -176,10 +187,9 @@ __global__ void __launch_bounds__(kThreads, 1)
       bool ok = true;
       for (int ti = 0; ti < my_tiles && ok; ++ti) {
         const Tile tl = nth_tile(p, cta, grid, ti);
-        const int n_kb = tl.is_gw ? p.num_kb_w : p.num_kb_x;
         const int bn = tl.is_gw ? p.BNw : p.BNx;
         const uint32_t tx = static_cast<uint32_t>(kABytes + bn * BK * 2);
-        for (int kb = 0; kb < n_kb; ++kb) {
+        for (int kb = tl.kb0; kb < tl.kb0 + tl.n_kb; ++kb) {
           const int s = static_cast<int>(it % kStages);
           if (!ptx::mbar_wait(&empty_bar[s], ((it / kStages) + 1) & 1u, p.status, (4u << 16) | 1u)) {
             ok = false;
@@ -217,7 +227,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       for (int ti = 0; ti < my_tiles && ok; ++ti) {
         const Tile tl = nth_tile(p, cta, grid, ti);
         const int slot = ti & 1;
-        const int n_kb = tl.is_gw ? p.num_kb_w : p.num_kb_x;
+        const int n_kb = tl.n_kb;
         const uint32_t d_tmem = tmem_base + slot * kSlotCols;
         const uint32_t idesc = tl.is_gw ? idesc_w : idesc_x;
         const uint32_t uses = static_cast<uint32_t>(ti >> 1);   // earlier uses of this slot
@@ -289,7 +299,15 @@ __global__ void __launch_bounds__(kThreads, 1)
           }
           if (row < p.Cout) {
             const long long colb = static_cast<long long>(tl.b) * bn + c0;
-            if (p.gw_bf16) {
+            if (p.gw_splits > 1) {
+              // K slice: fp32 partial plane, summed by the reduce kernel that follows
+              float* d = p.gw_planes + (static_cast<long long>(tl.slice) * p.Cout + row) * p.Cin;
+#pragma unroll
+              for (int q = 0; q < 32; q += 4) {
+                if (colb + q < p.Cin)
+                  *reinterpret_cast<uint4*>(d + colb + q) = make_uint4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+              }
+            } else if (p.gw_bf16) {
               __nv_bfloat16* d = static_cast<__nv_bfloat16*>(p.g_W) + row * p.Cin;
 #pragma unroll
               for (int q = 0; q < 32; q += 8) {
@@ -456,6 +474,19 @@ size_t fused_scratch_bytes(const lbp_layer& L, int r, FusedLayout* lay) {
   l.gy_hat = off;
   off += static_cast<size_t>(G) * 128 * L.Cout * 2;
   off = (off + 1023) / 1024 * 1024;
+  // fp32 planes for K slices of g_W: only layers with few GW tiles slice, and
+  // slices * tiles stays below the SM count (bounded here for up to 256 SMs)
+  l.planes = off;
+  {
+    const long long tiles_min = ((L.Cout + 127) / 128) * ((L.Cin + 255) / 256);
+    long long s_cap = tiles_min >= 96 ? 1 : 192 / tiles_min;
+    if (s_cap > 2 * G) s_cap = 2 * G;
+    l.planes_bytes = s_cap > 1 ? static_cast<size_t>(s_cap) * L.Cout * L.Cin * 4 : 0;
+    const size_t cap = 48u << 20;
+    if (l.planes_bytes > cap) l.planes_bytes = cap;
+  }
+  off += l.planes_bytes;
+  off = (off + 1023) / 1024 * 1024;
   l.trace = off;
   off += kFusedTraceBytes;
   l.total = (off + 1023) / 1024 * 1024;
@@ -493,37 +524,95 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
   p.mt_w = (L.Cout + 127) / 128;
   p.num_kb_w = p.G * (BM / BK);
   const int cin64 = (L.Cin + 63) / 64 * 64;
+  const int max_splits_by_ws =
+      static_cast<int>(lay.planes_bytes / (static_cast<size_t>(L.Cout) * L.Cin * 4));
+  // the search costs tens of microseconds of host time: remember recent answers
+  struct PlanKey {
+    int Cin, Cout, G, sms, max_splits;
+    int BNw, BNx, splits, kbps;
+  };
+  static thread_local PlanKey plan_cache[16];
+  static thread_local int plan_cache_n = 0, plan_cache_next = 0;
+  bool cached = false;
+  for (int i = 0; i < plan_cache_n; ++i) {
+    const PlanKey& c = plan_cache[i];
+    if (c.Cin == L.Cin && c.Cout == L.Cout && c.G == p.G && c.sms == sms &&
+        c.max_splits == max_splits_by_ws) {
+      p.BNw = c.BNw;
+      p.BNx = c.BNx;
+      p.gw_splits = c.splits;
+      p.kb_per_split_w = c.kbps;
+      cached = true;
+      break;
+    }
+  }
+  if (!cached) {
   double best = -1.0;
+  static const int kSplitChoices[] = {1, 2, 3, 4, 6, 8, 12, 16, 24, 32, 48, 64, 96, 128, 192};
   for (int bnw = 64; bnw <= 256; bnw += 64) {
     for (int bnx = 64; bnx <= 256; bnx += 64) {
       if (bnw > cin64 || bnx > cin64) continue;
-      const int nt_w = (L.Cin + bnw - 1) / bnw, n_tx = (L.Cin + bnx - 1) / bnx;
-      const int n_gw = p.mt_w * nt_w, n_gx = p.G * n_tx;
-      const double gw_cost = static_cast<double>(p.num_kb_w) * (kABytes + bnw * 128.0);
-      const double gx_cost = static_cast<double>(p.num_kb_x) * (kABytes + bnx * 128.0) +
-                             6000.0 * bnx;   // plus the expansion of the tile
-      const int total = n_gw + n_gx;
-      const int grid = total < sms ? total : sms;
-      double worst = 0.0;
-      for (int c = 0; c < grid; ++c) {
-        double load = 0.0;
-        for (int round = 0; round * grid < total; ++round) {
-          const int t = round * grid + ((round & 1) ? grid - 1 - c : c);
-          if (t < total) load += t < n_gw ? gw_cost : gx_cost;
+      for (int want : kSplitChoices) {
+        if (want > 1 && (want > max_splits_by_ws || want > p.num_kb_w / 4)) continue;
+        const int kbps = (p.num_kb_w + want - 1) / want;
+        const int splits = (p.num_kb_w + kbps - 1) / kbps;
+        const int nt_w = (L.Cin + bnw - 1) / bnw, n_tx = (L.Cin + bnx - 1) / bnx;
+        const int n_gw = p.mt_w * nt_w * splits, n_gx = p.G * n_tx;
+        const double gw_cost = static_cast<double>(kbps) * (kABytes + bnw * 128.0) + 1500.0 * bnw;
+        const double gx_cost = static_cast<double>(p.num_kb_x) * (kABytes + bnx * 128.0) +
+                               6000.0 * bnx;   // plus the expansion of the tile
+        const int total = n_gw + n_gx;
+        const int grid = total < sms ? total : sms;
+        double worst = 0.0;
+        for (int c = 0; c < grid; ++c) {
+          double load = 0.0;
+          for (int round = 0; round * grid < total; ++round) {
+            const int t = round * grid + ((round & 1) ? grid - 1 - c : c);
+            if (t < total) load += t < n_gw ? gw_cost : gx_cost;
+          }
+          if (load > worst) worst = load;
         }
-        if (load > worst) worst = load;
-      }
-      if (best < 0 || worst < best) {
-        best = worst;
-        p.BNw = bnw;
-        p.BNx = bnx;
+        if (splits > 1) {
+          // the reduce launch that follows: fixed cost plus its plane traffic at HBM
+          // speed, in the same unit (bytes a CTA ingests at ~100 GB/s)
+          const double plane_bytes = static_cast<double>(L.Cout) * L.Cin * 4.0;
+          worst += 600000.0 + (splits + 1.0) * plane_bytes / 40.0;
+        }
+        if (best < 0 || worst < best) {
+          best = worst;
+          p.BNw = bnw;
+          p.BNx = bnx;
+          p.gw_splits = splits;
+          p.kb_per_split_w = kbps;
+        }
       }
     }
   }
+    PlanKey& c = plan_cache[plan_cache_next];
+    c = PlanKey{L.Cin, L.Cout, p.G, sms, max_splits_by_ws, p.BNw, p.BNx, p.gw_splits, p.kb_per_split_w};
+    plan_cache_next = (plan_cache_next + 1) % 16;
+    if (plan_cache_n < 16) ++plan_cache_n;
+  }
+  // tuning overrides: LBP_FUSED_TILES="BNw,BNx,splits"
+  if (const char* e = std::getenv("LBP_FUSED_TILES")) {
+    int bw = 0, bx = 0, sp = 0;
+    if (sscanf(e, "%d,%d,%d", &bw, &bx, &sp) == 3 && bw >= 64 && bw <= 256 && bw % 64 == 0 &&
+        bx >= 64 && bx <= 256 && bx % 64 == 0 && sp >= 1 && (sp == 1 || sp <= max_splits_by_ws)) {
+      p.BNw = bw;
+      p.BNx = bx;
+      p.kb_per_split_w = (p.num_kb_w + sp - 1) / sp;
+      p.gw_splits = (p.num_kb_w + p.kb_per_split_w - 1) / p.kb_per_split_w;
+    }
+  }
+  if (const char* e = std::getenv("LBP_FUSED_VERBOSE"))
+    if (e[0] == '1')
+      fprintf(stderr, "lbp products: G=%d BNw=%d BNx=%d gw_splits=%d kb/split=%d\n", p.G, p.BNw, p.BNx,
+              p.gw_splits, p.kb_per_split_w);
   p.n_tx = (L.Cin + p.BNx - 1) / p.BNx;
   p.nt_w = (L.Cin + p.BNw - 1) / p.BNw;
   p.n_gx_tiles = p.G * p.n_tx;
-  p.n_gw_tiles = p.mt_w * p.nt_w;
+  p.n_gw_tiles = p.mt_w * p.nt_w * p.gw_splits;
+  p.gw_planes = reinterpret_cast<float*>(scratch + lay.planes);
   p.gw_bf16 = L.gw_dtype == LBP_BF16 ? 1 : 0;
   p.scale = 1.0f / static_cast<float>(K);
   p.x_hat = reinterpret_cast<__nv_bfloat16*>(scratch + lay.x_hat);
@@ -576,6 +665,9 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
     LBP_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tm_gyhat_k, tm_gyhat_mn, tm_xhat, tm_w, p, fb));
     count_launch();
     LBP_CUDA_TRY(cudaGetLastError());
+    if (p.gw_splits > 1)
+      return launch_splitk_reduce(p.gw_planes, g_W, static_cast<long long>(L.Cout) * L.Cin,
+                                  p.gw_splits, p.gw_bf16 != 0, stream);
     return LBP_OK;
   };
   switch (K * 100 + bp.LB) {

@@ -18,7 +18,9 @@ struct FusedParams {
   // products
   int32_t BNx, n_tx, num_kb_x;            // GX: column tile, tiles per row group, k-blocks (Cout / 64)
   int32_t BNw, mt_w, nt_w, num_kb_w;      // GW: 128 x BNw tiles, k-blocks (G * 2)
-  int32_t n_gx_tiles, n_gw_tiles;
+  int32_t n_gx_tiles, n_gw_tiles;         // n_gw_tiles counts K slices: mt_w * nt_w * gw_splits
+  int32_t gw_splits, kb_per_split_w;      // K slices of a GW tile (fp32 planes, reduced afterwards)
+  float* gw_planes;                       // [gw_splits][Cout][Cin] when gw_splits > 1
   int32_t gw_bf16;
   float scale;                            // 1/k
   __nv_bfloat16* x_hat;
@@ -36,7 +38,7 @@ struct FusedBasis {
 constexpr size_t kFusedTraceBytes = 256 * 8 * 8;   // last bytes of the scratch region
 
 struct FusedLayout {
-  size_t x_hat, gy_hat, trace, total;
+  size_t x_hat, gy_hat, planes, planes_bytes, trace, total;
   int G, bpt;
 };
 

@@ -101,6 +101,9 @@ int launch_gemm(const void* A, bool a_mn_major, const void* Bm, void* D, int in_
                 long long M, long long N, long long K, float* splitk_ws, size_t splitk_ws_bytes,
                 uint32_t* status, cudaStream_t stream);
 size_t gemm_splitk_ws_bytes(long long M, long long N, long long K, int in_dtype);
+// D[i] = sum over `splits` fp32 planes of mn elements each (mn a multiple of 4), in plane order.
+int launch_splitk_reduce(const float* planes, void* D, long long mn, int splits, bool d_bf16,
+                         cudaStream_t stream);
 
 int check_device_arch();
 
