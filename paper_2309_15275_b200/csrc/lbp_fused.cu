@@ -35,12 +35,13 @@ constexpr int kBBytes = 256 * BK * 2;            // 32 KB (up to 256 columns)
 constexpr int kStageBytes = kABytes + kBBytes;   // 48 KB
 constexpr int kChunkBytes = 64 * BK * 2;         // 8 KB: one 64-wide chunk of an MN-major tile
 constexpr int kEStride = 32;   // fp32 words per staged row; 16-byte chunk c of row i sits at chunk c ^ (i & 7)
-constexpr int kEBytes = BM * kEStride * 4;
+constexpr int kEBytes = (BM + 1) * kEStride * 4;   // 128 staged rows + one row of zeros
 constexpr int kEGroups = 2;                      // epilogue groups of 4 warps (one per TMEM lane quarter)
 constexpr int kThreads = (2 + 4 * kEGroups) * 32;
 constexpr int kOffE = kStages * kStageBytes;
 constexpr int kOffBar = kOffE + kEGroups * kEBytes;
 constexpr int kSmemBytes = kOffBar + 256 + 1024;
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA exceeded");
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kSlotCols = 256;   // two accumulator slots; tile number t of a CTA uses slot t & 1
 
@@ -270,6 +271,10 @@ __global__ void __launch_bounds__(kThreads, 1)
     const uint32_t lane_bits = static_cast<uint32_t>(quarter * 32) << 16;
     float* const Eg = E + eg * (kEBytes / 4);
     const int bar_id = 1 + eg;
+    // row 128 stays zero: unselected coefficients are gathered from there, which
+    // keeps the gather free of branches
+    if (etid < kEStride) Eg[BM * kEStride + etid] = 0.f;
+    named_bar_sync(bar_id, 128);
     for (int ti = 0; ti < my_tiles; ++ti) {
       const Tile tl = nth_tile(p, cta, grid, ti);
       const int slot = ti & 1;
@@ -368,25 +373,21 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
                 for (int b = 0; b < LB; ++b) {
                   const int q = fb.qmap[a * LB + b];
-                  const int row_q = row_b + q;
+                  const int row_q = q >= 0 ? row_b + q : BM;
                   if constexpr (NCH == 4) {
-                    float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (q >= 0)
-                      f = *reinterpret_cast<const float4*>(Eg + row_q * kEStride + ((cc ^ (row_q & 7)) << 2));
+                    const float4 f =
+                        *reinterpret_cast<const float4*>(Eg + row_q * kEStride + ((cc ^ (row_q & 7)) << 2));
                     acc[a][b][0] = f.x;
                     acc[a][b][1] = f.y;
                     acc[a][b][2] = f.z;
                     acc[a][b][3] = f.w;
                   } else if constexpr (NCH == 2) {
-                    float2 f = make_float2(0.f, 0.f);
-                    if (q >= 0)
-                      f = *reinterpret_cast<const float2*>(Eg + row_q * kEStride +
-                                                           (((cc >> 1) ^ (row_q & 7)) << 2) + (cc & 1) * 2);
+                    const float2 f = *reinterpret_cast<const float2*>(
+                        Eg + row_q * kEStride + (((cc >> 1) ^ (row_q & 7)) << 2) + (cc & 1) * 2);
                     acc[a][b][0] = f.x;
                     acc[a][b][1] = f.y;
                   } else {
-                    acc[a][b][0] =
-                        q >= 0 ? Eg[row_q * kEStride + (((cc >> 2) ^ (row_q & 7)) << 2) + (cc & 3)] : 0.f;
+                    acc[a][b][0] = Eg[row_q * kEStride + (((cc >> 2) ^ (row_q & 7)) << 2) + (cc & 3)];
                   }
                 }
               }
