@@ -21,6 +21,7 @@
 #include <cstdlib>
 
 #include "lbp_fused.cuh"
+#include "lbp_fused_epilogue.cuh"
 #include "lbp_internal.h"
 #include "ptx_sm100.cuh"
 #include "wht_device.cuh"
@@ -28,15 +29,12 @@
 namespace lbp {
 namespace fused {
 
-constexpr int BM = 128, BK = 64;
+constexpr int BK = 64;
 constexpr int kStages = 4;
 constexpr int kABytes = BM * BK * 2;             // 16 KB
 constexpr int kBBytes = 256 * BK * 2;            // 32 KB (up to 256 columns)
 constexpr int kStageBytes = kABytes + kBBytes;   // 48 KB
 constexpr int kChunkBytes = 64 * BK * 2;         // 8 KB: one 64-wide chunk of an MN-major tile
-constexpr int kEStride = 32;   // fp32 words per staged row; 16-byte chunk c of row i sits at chunk c ^ (i & 7)
-constexpr int kEBytes = (BM + 1) * kEStride * 4;   // 128 staged rows + one row of zeros
-constexpr int kEGroups = 2;                      // epilogue groups of 4 warps (one per TMEM lane quarter)
 constexpr int kThreads = (2 + 4 * kEGroups) * 32;
 constexpr int kOffE = kStages * kStageBytes;
 constexpr int kOffBar = kOffE + kEGroups * kEBytes;
@@ -45,9 +43,6 @@ static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA exceede
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kSlotCols = 256;   // two accumulator slots; tile number t of a CTA uses slot t & 1
 
-__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
-}
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -67,14 +62,11 @@ __device__ __forceinline__ void trace_mark(const FusedParams& p, int slot, bool 
   }
 }
 
-__device__ __forceinline__ int blocks_in_group(const FusedParams& p, int g) {
-  const int left = p.nb - g * p.bpt;
-  return left < p.bpt ? left : p.bpt;
-}
-
 // Tile list.  Tiles are numbered with the GW tiles (the larger ones) first and
 // dealt to the CTAs in a snake: round 0 forwards, round 1 backwards, ... so
-// that a CTA that got a large tile gets its next one last.
+// that a CTA that got a large tile gets its next one last.  A CTA works through
+// its list backwards: GX tiles (long expansion epilogue) first, its GW tile (short
+// epilogue) last, so that little is left to do after the last MMA.
 struct Tile {
   int is_gw;
   int a, b;          // GW: (i, j) ; GX: (m, n)
@@ -268,7 +260,6 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int ew = (warp - 2) & 3;           // warp within the group
     const int quarter = warp & 3;            // TMEM lane quarter this warp may read
     const int etid = ew * 32 + lane;         // 0..127 within the group
-    const uint32_t lane_bits = static_cast<uint32_t>(quarter * 32) << 16;
     float* const Eg = E + eg * (kEBytes / 4);
     const int bar_id = 1 + eg;
     // row 128 stays zero: unselected coefficients are gathered from there, which
@@ -286,161 +277,17 @@ __global__ void __launch_bounds__(kThreads, 1)
       if (*abort_flag) break;
       ptx::tc_fence_after_sync();
       if (etid == 0 && eg == 0) trace_mark(p, 5, true);
-      const int bn = tl.is_gw ? p.BNw : p.BNx;
-      bool released = false;
-
-      if (tl.is_gw) {
-        // ---- GW tile: g_W[128 i + row, BNw j + col] ----
-        const long long row = static_cast<long long>(tl.a) * 128 + quarter * 32 + lane;
-        for (int c0 = eg * 32; c0 < bn; c0 += 32 * kEGroups) {
-          uint32_t v[32];
-          ptx::tmem_ld_32x32(tmem_base + lane_bits + acc_col + c0, v);
-          ptx::tmem_ld_wait();
-          if (c0 + 32 * kEGroups >= bn) {
-            released = true;
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&acc_empty[slot]);
-          }
-          if (row < p.Cout) {
-            const long long colb = static_cast<long long>(tl.b) * bn + c0;
-            if (p.gw_splits > 1) {
-              // K slice: fp32 partial plane, summed by the reduce kernel that follows
-              float* d = p.gw_planes + (static_cast<long long>(tl.slice) * p.Cout + row) * p.Cin;
-#pragma unroll
-              for (int q = 0; q < 32; q += 4) {
-                if (colb + q < p.Cin)
-                  *reinterpret_cast<uint4*>(d + colb + q) = make_uint4(v[q], v[q + 1], v[q + 2], v[q + 3]);
-              }
-            } else if (p.gw_bf16) {
-              __nv_bfloat16* d = static_cast<__nv_bfloat16*>(p.g_W) + row * p.Cin;
-#pragma unroll
-              for (int q = 0; q < 32; q += 8) {
-                if (colb + q < p.Cin) {
-                  uint4 o;
-                  o.x = pack_bf16x2(__uint_as_float(v[q]), __uint_as_float(v[q + 1]));
-                  o.y = pack_bf16x2(__uint_as_float(v[q + 2]), __uint_as_float(v[q + 3]));
-                  o.z = pack_bf16x2(__uint_as_float(v[q + 4]), __uint_as_float(v[q + 5]));
-                  o.w = pack_bf16x2(__uint_as_float(v[q + 6]), __uint_as_float(v[q + 7]));
-                  *reinterpret_cast<uint4*>(d + colb + q) = o;
-                }
-              }
-            } else {
-              float* d = static_cast<float*>(p.g_W) + row * p.Cin;
-#pragma unroll
-              for (int q = 0; q < 32; q += 4) {
-                if (colb + q < p.Cin)
-                  *reinterpret_cast<uint4*>(d + colb + q) = make_uint4(v[q], v[q + 1], v[q + 2], v[q + 3]);
-              }
-            }
-          }
-        }
-      } else {
-        // ---- GX tile: expand g_x_hat (128 rows x BNx columns) into g_x ----
-        const int m = tl.a, n = tl.b;
-        const int bg = blocks_in_group(p, m);
-        // channels per thread (the 8 x 8 array of order 8 leaves registers for one)
-        constexpr int NCH = LB <= 4 ? 4 : (K >= 16 ? 2 : 1);
-        constexpr int RUN = K / LB;
-        constexpr int CPT = 32 / NCH;       // threads across one 32-column chunk
-        constexpr int BSLOTS = 128 / CPT;   // blocks expanded concurrently
-        const int cc = etid % CPT, bs = etid / CPT;
-        // element offsets of a token inside a block fit 32 bits (checked on the host)
-        const int tok_stride = p.Cin, row_stride = p.W * p.Cin;
-        for (int c0 = eg * 32; c0 < bn; c0 += 32 * kEGroups) {
-          uint32_t v[32];
-          ptx::tmem_ld_32x32(tmem_base + lane_bits + acc_col + c0, v);
-          ptx::tmem_ld_wait();
-          if (c0 + 32 * kEGroups >= bn) {
-            released = true;
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&acc_empty[slot]);
-          }
-          const int erow_i = quarter * 32 + lane;
-          uint4* erow = reinterpret_cast<uint4*>(Eg + erow_i * kEStride);
-#pragma unroll
-          for (int q = 0; q < 8; ++q)
-            erow[q ^ (erow_i & 7)] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-          named_bar_sync(bar_id, 128);
-          const int ch = n * bn + c0 + cc * NCH;
-          if (ch < p.Cin) {
-            for (int bl = bs; bl < bg; bl += BSLOTS) {
-              float acc[LB][LB][NCH];
-              const int row_b = bl * p.r;
-#pragma unroll
-              for (int a = 0; a < LB; ++a) {
-#pragma unroll
-                for (int b = 0; b < LB; ++b) {
-                  const int q = fb.qmap[a * LB + b];
-                  const int row_q = q >= 0 ? row_b + q : BM;
-                  if constexpr (NCH == 4) {
-                    const float4 f =
-                        *reinterpret_cast<const float4*>(Eg + row_q * kEStride + ((cc ^ (row_q & 7)) << 2));
-                    acc[a][b][0] = f.x;
-                    acc[a][b][1] = f.y;
-                    acc[a][b][2] = f.z;
-                    acc[a][b][3] = f.w;
-                  } else if constexpr (NCH == 2) {
-                    const float2 f = *reinterpret_cast<const float2*>(
-                        Eg + row_q * kEStride + (((cc >> 1) ^ (row_q & 7)) << 2) + (cc & 1) * 2);
-                    acc[a][b][0] = f.x;
-                    acc[a][b][1] = f.y;
-                  } else {
-                    acc[a][b][0] = Eg[row_q * kEStride + (((cc >> 2) ^ (row_q & 7)) << 2) + (cc & 3)];
-                  }
-                }
-              }
-              hadamard_rows<LB, NCH>(acc);
-              hadamard_cols<LB, NCH>(acc);
-              const int blk = m * p.bpt + bl;
-              const int bw = blk % p.Wb, t2 = blk / p.Wb, bh = t2 % p.Hb, b = t2 / p.Hb;
-              __nv_bfloat16* o = p.g_x +
-                                 ((static_cast<long long>(b) * p.H + bh * K) * p.W + bw * K) * p.Cin + ch;
-              // each of the LB x LB values covers a RUN x RUN patch of tokens: scale,
-              // round and pack once, store RUN * RUN times
-#pragma unroll
-              for (int a = 0; a < LB; ++a) {
-#pragma unroll
-                for (int b2 = 0; b2 < LB; ++b2) {
-                  if constexpr (NCH == 4) {
-                    uint2 pk;
-                    pk.x = pack_bf16x2(acc[a][b2][0] * p.scale, acc[a][b2][1] * p.scale);
-                    pk.y = pack_bf16x2(acc[a][b2][2] * p.scale, acc[a][b2][3] * p.scale);
-#pragma unroll
-                    for (int du = 0; du < RUN; ++du)
-#pragma unroll
-                      for (int dv = 0; dv < RUN; ++dv)
-                        *reinterpret_cast<uint2*>(o + (a * RUN + du) * row_stride +
-                                                  (b2 * RUN + dv) * tok_stride) = pk;
-                  } else if constexpr (NCH == 1) {
-                    const __nv_bfloat16 hv = __float2bfloat16_rn(acc[a][b2][0] * p.scale);
-#pragma unroll
-                    for (int du = 0; du < RUN; ++du)
-#pragma unroll
-                      for (int dv = 0; dv < RUN; ++dv)
-                        o[(a * RUN + du) * row_stride + (b2 * RUN + dv) * tok_stride] = hv;
-                  } else {
-                    const uint32_t pk = pack_bf16x2(acc[a][b2][0] * p.scale, acc[a][b2][1] * p.scale);
-#pragma unroll
-                    for (int du = 0; du < RUN; ++du)
-#pragma unroll
-                      for (int dv = 0; dv < RUN; ++dv)
-                        *reinterpret_cast<uint32_t*>(o + (a * RUN + du) * row_stride +
-                                                     (b2 * RUN + dv) * tok_stride) = pk;
-                  }
-                }
-              }
-            }
-          }
-          named_bar_sync(bar_id, 128);
-        }
-      }
-      if (!released) {   // this group had no chunk of the tile
-        ptx::tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&acc_empty[slot]);
-      }
+      DrainTile dt;
+      dt.is_gw = tl.is_gw;
+      dt.row_base = tl.a * 128;
+      dt.group = tl.a;
+      dt.col_base = tl.b * (tl.is_gw ? p.BNw : p.BNx);
+      dt.bn = tl.is_gw ? p.BNw : p.BNx;
+      dt.slice = tl.slice;
+      dt.tmem_acc = tmem_base + acc_col;
+      uint64_t* release_bar = &acc_empty[slot];
+      drain_tile<K, LB>(p, fb, dt, Eg, bar_id, eg, etid, quarter, lane,
+                        [release_bar]() { ptx::mbar_arrive(release_bar); });
     }
     if (etid == 0) trace_mark(p, 4);   // latest of the groups
   }
@@ -518,6 +365,24 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
   p.G = lay.G;
   p.Cin = L.Cin;
   p.Cout = L.Cout;
+  p.gw_bf16 = L.gw_dtype == LBP_BF16 ? 1 : 0;
+  p.scale = 1.0f / static_cast<float>(K);
+  p.x_hat = reinterpret_cast<__nv_bfloat16*>(scratch + lay.x_hat);
+  p.gy_hat = reinterpret_cast<__nv_bfloat16*>(scratch + lay.gy_hat);
+  p.gw_planes = reinterpret_cast<float*>(scratch + lay.planes);
+  p.g_x = static_cast<__nv_bfloat16*>(g_x);
+  p.g_W = g_W;
+  p.status = status;
+  p.trace = nullptr;
+  p.num_kb_x = (L.Cout + BK - 1) / BK;
+  p.num_kb_w = p.G * (BM / BK);
+  FusedBasis fb;
+  for (int n = 0; n < 64; ++n) fb.qmap[n] = -1;
+  for (int a = 0; a < bp.LB; ++a)
+    for (int b = 0; b < bp.LB; ++b) fb.qmap[a * bp.LB + b] = bp.qmap[a * bp.LB + b];
+  if (fused_pair_supported(L, sms))
+    return launch_fused_pair(x, g_y, W, g_W, L, bp, p, fb, lay, sms, status, stream, hook, hook_arg);
+
   // Column tiles are multiples of 64 (one TMA chunk) up to 256.  Each
   // candidate pair is scored by the operand bytes of the busiest CTA under the
   // snake assignment of the tile list (the kernel is bound by operand traffic).
@@ -628,11 +493,6 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
       LBP_CUDA_TRY(cudaMemsetAsync(p.trace, 0, kFusedTraceBytes, stream));
     }
   }
-
-  FusedBasis fb;
-  for (int n = 0; n < 64; ++n) fb.qmap[n] = -1;
-  for (int a = 0; a < bp.LB; ++a)
-    for (int b = 0; b < bp.LB; ++b) fb.qmap[a * bp.LB + b] = bp.qmap[a * bp.LB + b];
 
   // Algorithm 1, steps 1-2: x_hat and g_y_hat, rows padded to 128-row groups
   if (int e = launch_project2(g_y, p.gy_hat, L.Cout, x, p.x_hat, L.Cin, LBP_BF16, L.B, L.H, L.W, bp,

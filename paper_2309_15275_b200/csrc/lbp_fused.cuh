@@ -51,4 +51,11 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
                  const lbp_layer& L, const BasisPlan& bp, uint8_t* scratch, uint32_t* status,
                  cudaStream_t stream, FusedPhaseHook hook, void* hook_arg);
 
+// CTA-pair variant (tcgen05 cta_group::2): used when Cin >= 128 and the SM count is even.
+bool fused_pair_supported(const lbp_layer& L, int sms);
+int launch_fused_pair(const void* x, const void* g_y, const void* W, void* g_W, const lbp_layer& L,
+                      const BasisPlan& bp, FusedParams p, const FusedBasis& fb,
+                      const FusedLayout& lay, int sms, uint32_t* status, cudaStream_t stream,
+                      FusedPhaseHook hook, void* hook_arg);
+
 }  // namespace lbp

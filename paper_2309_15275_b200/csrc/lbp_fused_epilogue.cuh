@@ -1,0 +1,212 @@
+// Epilogue of one accumulator tile of the products kernels, shared by the
+// one-CTA and the CTA-pair variants: a GW tile is written to g_W (or to an fp32
+// K-slice plane); a GX tile is expanded with the transposed bases (Eq. 7) and
+// written to g_x, so g_x_hat never leaves the chip.
+//
+// Four warps (one per TMEM lane quarter) form a group; group `eg` takes the
+// 32-column chunks eg, eg + kEGroups, ... of the tile.  A chunk goes TMEM ->
+// registers -> swizzled shared staging (row = low-rank row, 32 columns); then
+// every thread owns NCH channels of one block, gathers that block's r
+// coefficients, runs the LB x LB butterfly and stores the k x k tokens.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "lbp_fused.cuh"
+#include "ptx_sm100.cuh"
+#include "wht_device.cuh"
+
+namespace lbp {
+namespace fused {
+
+constexpr int BM = 128;
+constexpr int kEStride = 32;   // fp32 words per staged row; 16-byte chunk c of row i sits at chunk c ^ (i & 7)
+constexpr int kEBytes = (BM + 1) * kEStride * 4;   // 128 staged rows + one row of zeros
+constexpr int kEGroups = 2;                        // epilogue groups of 4 warps
+
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+__device__ __forceinline__ int blocks_in_group(const FusedParams& p, int g) {
+  const int left = p.nb - g * p.bpt;
+  return left < p.bpt ? left : p.bpt;
+}
+
+// What the epilogue needs to know about the accumulator it drains.
+struct DrainTile {
+  int is_gw;
+  int row_base;       // GW: first g_W row of these 128 accumulator rows
+  int group;          // GX: 128-row group of low-rank rows
+  int col_base;       // first output column (channel) of the tile
+  int bn;             // accumulator columns in use
+  int slice;          // GW: K slice (plane index when gw_splits > 1)
+  uint32_t tmem_acc;  // TMEM address of column 0, lane 0 of the accumulator
+};
+
+// `release()` is called by lane 0 of every warp once the warp has read its last
+// accumulator column (the tensor core may then overwrite the slot).
+template <int K, int LB, class Release>
+__device__ __forceinline__ void drain_tile(const FusedParams& p, const FusedBasis& fb,
+                                           const DrainTile& t, float* Eg, int bar_id, int eg,
+                                           int etid, int quarter, int lane, Release release) {
+  const uint32_t lane_bits = static_cast<uint32_t>(quarter * 32) << 16;
+  bool released = false;
+
+  if (t.is_gw) {
+    // ---- GW tile: g_W[128 i + row, BNw j + col] ----
+    const long long row = static_cast<long long>(t.row_base) + quarter * 32 + lane;
+    for (int c0 = eg * 32; c0 < t.bn; c0 += 32 * kEGroups) {
+      uint32_t v[32];
+      ptx::tmem_ld_32x32(t.tmem_acc + lane_bits + c0, v);
+      ptx::tmem_ld_wait();
+      if (c0 + 32 * kEGroups >= t.bn) {
+        released = true;
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) release();
+      }
+      if (row < p.Cout) {
+        const long long colb = static_cast<long long>(t.col_base) + c0;
+        if (p.gw_splits > 1) {
+          // K slice: fp32 partial plane, summed by the reduce kernel that follows
+          float* d = p.gw_planes + (static_cast<long long>(t.slice) * p.Cout + row) * p.Cin;
+#pragma unroll
+          for (int q = 0; q < 32; q += 4) {
+            if (colb + q < p.Cin)
+              *reinterpret_cast<uint4*>(d + colb + q) = make_uint4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+          }
+        } else if (p.gw_bf16) {
+          __nv_bfloat16* d = static_cast<__nv_bfloat16*>(p.g_W) + row * p.Cin;
+#pragma unroll
+          for (int q = 0; q < 32; q += 8) {
+            if (colb + q < p.Cin) {
+              uint4 o;
+              o.x = pack_bf16x2(__uint_as_float(v[q]), __uint_as_float(v[q + 1]));
+              o.y = pack_bf16x2(__uint_as_float(v[q + 2]), __uint_as_float(v[q + 3]));
+              o.z = pack_bf16x2(__uint_as_float(v[q + 4]), __uint_as_float(v[q + 5]));
+              o.w = pack_bf16x2(__uint_as_float(v[q + 6]), __uint_as_float(v[q + 7]));
+              *reinterpret_cast<uint4*>(d + colb + q) = o;
+            }
+          }
+        } else {
+          float* d = static_cast<float*>(p.g_W) + row * p.Cin;
+#pragma unroll
+          for (int q = 0; q < 32; q += 4) {
+            if (colb + q < p.Cin)
+              *reinterpret_cast<uint4*>(d + colb + q) = make_uint4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+          }
+        }
+      }
+    }
+  } else {
+    // ---- GX tile: expand g_x_hat (128 rows x BNx columns) into g_x ----
+    const int m = t.group;
+    const int bg = blocks_in_group(p, m);
+    // channels per thread (the 8 x 8 array of order 8 leaves registers for one)
+    constexpr int NCH = LB <= 4 ? 4 : (K >= 16 ? 2 : 1);
+    constexpr int RUN = K / LB;
+    constexpr int CPT = 32 / NCH;       // threads across one 32-column chunk
+    constexpr int BSLOTS = 128 / CPT;   // blocks expanded concurrently
+    const int cc = etid % CPT, bs = etid / CPT;
+    // element offsets of a token inside a block fit 32 bits (checked on the host)
+    const int tok_stride = p.Cin, row_stride = p.W * p.Cin;
+    for (int c0 = eg * 32; c0 < t.bn; c0 += 32 * kEGroups) {
+      uint32_t v[32];
+      ptx::tmem_ld_32x32(t.tmem_acc + lane_bits + c0, v);
+      ptx::tmem_ld_wait();
+      if (c0 + 32 * kEGroups >= t.bn) {
+        released = true;
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) release();
+      }
+      const int erow_i = quarter * 32 + lane;
+      uint4* erow = reinterpret_cast<uint4*>(Eg + erow_i * kEStride);
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        erow[q ^ (erow_i & 7)] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+      named_bar_sync(bar_id, 128);
+      const int ch = t.col_base + c0 + cc * NCH;
+      if (ch < p.Cin) {
+        for (int bl = bs; bl < bg; bl += BSLOTS) {
+          float acc[LB][LB][NCH];
+          const int row_b = bl * p.r;
+#pragma unroll
+          for (int a = 0; a < LB; ++a) {
+#pragma unroll
+            for (int b = 0; b < LB; ++b) {
+              const int q = fb.qmap[a * LB + b];
+              const int row_q = q >= 0 ? row_b + q : BM;
+              if constexpr (NCH == 4) {
+                const float4 f =
+                    *reinterpret_cast<const float4*>(Eg + row_q * kEStride + ((cc ^ (row_q & 7)) << 2));
+                acc[a][b][0] = f.x;
+                acc[a][b][1] = f.y;
+                acc[a][b][2] = f.z;
+                acc[a][b][3] = f.w;
+              } else if constexpr (NCH == 2) {
+                const float2 f = *reinterpret_cast<const float2*>(
+                    Eg + row_q * kEStride + (((cc >> 1) ^ (row_q & 7)) << 2) + (cc & 1) * 2);
+                acc[a][b][0] = f.x;
+                acc[a][b][1] = f.y;
+              } else {
+                acc[a][b][0] = Eg[row_q * kEStride + (((cc >> 2) ^ (row_q & 7)) << 2) + (cc & 3)];
+              }
+            }
+          }
+          hadamard_rows<LB, NCH>(acc);
+          hadamard_cols<LB, NCH>(acc);
+          const int blk = m * p.bpt + bl;
+          const int bw = blk % p.Wb, t2 = blk / p.Wb, bh = t2 % p.Hb, b = t2 / p.Hb;
+          __nv_bfloat16* o = p.g_x +
+                             ((static_cast<long long>(b) * p.H + bh * K) * p.W + bw * K) * p.Cin + ch;
+          // each of the LB x LB values covers a RUN x RUN patch of tokens: scale,
+          // round and pack once, store RUN * RUN times
+#pragma unroll
+          for (int a = 0; a < LB; ++a) {
+#pragma unroll
+            for (int b2 = 0; b2 < LB; ++b2) {
+              if constexpr (NCH == 4) {
+                uint2 pk;
+                pk.x = pack_bf16x2(acc[a][b2][0] * p.scale, acc[a][b2][1] * p.scale);
+                pk.y = pack_bf16x2(acc[a][b2][2] * p.scale, acc[a][b2][3] * p.scale);
+#pragma unroll
+                for (int du = 0; du < RUN; ++du)
+#pragma unroll
+                  for (int dv = 0; dv < RUN; ++dv)
+                    *reinterpret_cast<uint2*>(o + (a * RUN + du) * row_stride +
+                                              (b2 * RUN + dv) * tok_stride) = pk;
+              } else if constexpr (NCH == 1) {
+                const __nv_bfloat16 hv = __float2bfloat16_rn(acc[a][b2][0] * p.scale);
+#pragma unroll
+                for (int du = 0; du < RUN; ++du)
+#pragma unroll
+                  for (int dv = 0; dv < RUN; ++dv)
+                    o[(a * RUN + du) * row_stride + (b2 * RUN + dv) * tok_stride] = hv;
+              } else {
+                const uint32_t pk = pack_bf16x2(acc[a][b2][0] * p.scale, acc[a][b2][1] * p.scale);
+#pragma unroll
+                for (int du = 0; du < RUN; ++du)
+#pragma unroll
+                  for (int dv = 0; dv < RUN; ++dv)
+                    *reinterpret_cast<uint32_t*>(o + (a * RUN + du) * row_stride +
+                                                 (b2 * RUN + dv) * tok_stride) = pk;
+              }
+            }
+          }
+        }
+      }
+      named_bar_sync(bar_id, 128);
+    }
+  }
+  if (!released) {   // this group had no chunk of the tile
+    ptx::tc_fence_before_sync();
+    __syncwarp();
+    if (lane == 0) release();
+  }
+}
+
+}  // namespace fused
+}  // namespace lbp
