@@ -64,9 +64,9 @@ __device__ __forceinline__ void trace_mark(const FusedParams& p, int slot, bool 
 
 // Tile list.  Tiles are numbered with the GW tiles (the larger ones) first and
 // dealt to the CTAs in a snake: round 0 forwards, round 1 backwards, ... so
-// that a CTA that got a large tile gets its next one last.  A CTA works through
-// its list backwards: GX tiles (long expansion epilogue) first, its GW tile (short
-// epilogue) last, so that little is left to do after the last MMA.
+// that a CTA that got a large tile gets its next one last.  A CTA takes its
+// tiles in list order (walking the list backwards, GX tiles first, measured no
+// faster).
 struct Tile {
   int is_gw;
   int a, b;          // GW: (i, j) ; GX: (m, n)

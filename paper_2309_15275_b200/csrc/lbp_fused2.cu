@@ -126,9 +126,8 @@ __device__ __forceinline__ void trace_mark(const FusedParams& p, int slot, bool 
   }
 }
 
-// ---- pair-tile list (same snake as the one-CTA kernel, over CTA pairs).  A pair
-// works through its list backwards: the GX tiles (long expansion epilogue) first,
-// the GW tile (short epilogue) last, so that little is left after the last MMA.
+// ---- pair-tile list (same snake as the one-CTA kernel, over CTA pairs), taken
+// in list order ----
 struct PairTile {
   int is_gw;
   int a, b;        // GW: (i, j) ; GX: (group pair, n)

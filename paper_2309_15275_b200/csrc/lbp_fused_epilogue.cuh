@@ -56,7 +56,9 @@ __device__ __forceinline__ void drain_tile(const FusedParams& p, const FusedBasi
 
   if (t.is_gw) {
     // ---- GW tile: g_W[128 i + row, BNw j + col] ----
-    const long long row = static_cast<long long>(t.row_base) + quarter * 32 + lane;
+    // A chunk is staged like a GX chunk and written out with eight lanes along a
+    // row, so that a store instruction covers whole 128-byte pieces of four rows.
+    const int ew = etid >> 5;
     for (int c0 = eg * 32; c0 < t.bn; c0 += 32 * kEGroups) {
       uint32_t v[32];
       ptx::tmem_ld_32x32(t.tmem_acc + lane_bits + c0, v);
@@ -67,38 +69,50 @@ __device__ __forceinline__ void drain_tile(const FusedParams& p, const FusedBasi
         __syncwarp();
         if (lane == 0) release();
       }
-      if (row < p.Cout) {
-        const long long colb = static_cast<long long>(t.col_base) + c0;
-        if (p.gw_splits > 1) {
-          // K slice: fp32 partial plane, summed by the reduce kernel that follows
-          float* d = p.gw_planes + (static_cast<long long>(t.slice) * p.Cout + row) * p.Cin;
+      const int erow_i = quarter * 32 + lane;
+      uint4* erow = reinterpret_cast<uint4*>(Eg + erow_i * kEStride);
 #pragma unroll
-          for (int q = 0; q < 32; q += 4) {
-            if (colb + q < p.Cin)
-              *reinterpret_cast<uint4*>(d + colb + q) = make_uint4(v[q], v[q + 1], v[q + 2], v[q + 3]);
-          }
-        } else if (p.gw_bf16) {
-          __nv_bfloat16* d = static_cast<__nv_bfloat16*>(p.g_W) + row * p.Cin;
+      for (int q = 0; q < 8; ++q)
+        erow[q ^ (erow_i & 7)] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+      named_bar_sync(bar_id, 128);
+      if (p.gw_splits > 1 || !p.gw_bf16) {
+        // fp32 g_W, or a K slice: fp32 partial plane, summed by the reduce kernel that follows
+        float* dst = p.gw_splits > 1
+                         ? p.gw_planes + static_cast<long long>(t.slice) * p.Cout * p.Cin
+                         : static_cast<float*>(p.g_W);
+        const int o = lane & 7, rs = lane >> 3;
+        const int col = t.col_base + c0 + o * 4;
 #pragma unroll
-          for (int q = 0; q < 32; q += 8) {
-            if (colb + q < p.Cin) {
-              uint4 o;
-              o.x = pack_bf16x2(__uint_as_float(v[q]), __uint_as_float(v[q + 1]));
-              o.y = pack_bf16x2(__uint_as_float(v[q + 2]), __uint_as_float(v[q + 3]));
-              o.z = pack_bf16x2(__uint_as_float(v[q + 4]), __uint_as_float(v[q + 5]));
-              o.w = pack_bf16x2(__uint_as_float(v[q + 6]), __uint_as_float(v[q + 7]));
-              *reinterpret_cast<uint4*>(d + colb + q) = o;
-            }
-          }
-        } else {
-          float* d = static_cast<float*>(p.g_W) + row * p.Cin;
+        for (int it = 0; it < 8; ++it) {
+          const int row = it * 16 + ew * 4 + rs;
+          const long long grow = static_cast<long long>(t.row_base) + row;
+          if (grow < p.Cout && col < p.Cin)
+            *reinterpret_cast<uint4*>(dst + grow * p.Cin + col) =
+                *reinterpret_cast<const uint4*>(Eg + row * kEStride + ((o ^ (row & 7)) << 2));
+        }
+      } else {
+        __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.g_W);
+        const int o = lane & 3, rs = lane >> 2;
+        const int col = t.col_base + c0 + o * 8;
 #pragma unroll
-          for (int q = 0; q < 32; q += 4) {
-            if (colb + q < p.Cin)
-              *reinterpret_cast<uint4*>(d + colb + q) = make_uint4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+        for (int it = 0; it < 4; ++it) {
+          const int row = it * 32 + ew * 8 + rs;
+          const long long grow = static_cast<long long>(t.row_base) + row;
+          if (grow < p.Cout && col < p.Cin) {
+            const float4 f0 = *reinterpret_cast<const float4*>(
+                Eg + row * kEStride + (((2 * o) ^ (row & 7)) << 2));
+            const float4 f1 = *reinterpret_cast<const float4*>(
+                Eg + row * kEStride + (((2 * o + 1) ^ (row & 7)) << 2));
+            uint4 pk;
+            pk.x = pack_bf16x2(f0.x, f0.y);
+            pk.y = pack_bf16x2(f0.z, f0.w);
+            pk.z = pack_bf16x2(f1.x, f1.y);
+            pk.w = pack_bf16x2(f1.z, f1.w);
+            *reinterpret_cast<uint4*>(dst + grow * p.Cin + col) = pk;
           }
         }
       }
+      named_bar_sync(bar_id, 128);
     }
   } else {
     // ---- GX tile: expand g_x_hat (128 rows x BNx columns) into g_x ----
