@@ -166,6 +166,9 @@ __global__ void __launch_bounds__(kThreads, 1)
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   if (threadIdx.x == 0) trace_mark(p, 0);
+  // the next kernel on the stream (the projection of the next call) may be
+  // scheduled as SMs free up; it waits for this grid before touching memory
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int my_tiles = tiles_of_cta(p, cta, grid);
 

@@ -231,6 +231,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 
   const int my_tiles = tiles_of_pair(p, pair, pairs);
   if (threadIdx.x == 0) trace_mark(p, 0);
+  // the next kernel on the stream (the projection of the next call) may be
+  // scheduled as SMs free up; it waits for this grid before touching memory
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (warp == 0) {
     // =========================== TMA producer (both CTAs) ===========================

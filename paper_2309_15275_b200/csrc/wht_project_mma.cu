@@ -97,6 +97,11 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
   // itself up as SMs free up; it still waits for this grid before reading
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   __syncthreads();
+  // this kernel itself may have been launched the same way behind an earlier
+  // kernel on the stream (the products kernel of the previous call, which still
+  // reads the buffers written below): nothing is read or written before that
+  // kernel has completed
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   const uint32_t first = blockIdx.x * NW + warp;
   const uint32_t stride = gridDim.x * NW;
@@ -238,7 +243,17 @@ static int launch_mma_one(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bf
   }
   const uint32_t want = (p.n_items + Cfg::kWarps - 1) / Cfg::kWarps;
   const int grid = static_cast<int>(want < static_cast<uint32_t>(sms) ? want : sms);
-  kern<<<grid, Cfg::kWarps * 32, Cfg::kSmemBytes, stream>>>(tmaps[0], tmaps[1], out0, out1, p, mp);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(Cfg::kWarps * 32);
+  cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  LBP_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmaps[0], tmaps[1], out0, out1, p, mp));
   count_launch();
   LBP_CUDA_TRY(cudaGetLastError());
   return LBP_OK;
