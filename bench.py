@@ -49,7 +49,7 @@ def _peaks():
 # DRAM traffic per step (sum over the four layers, bytes) of the two kernels, from
 # the ncu capture summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum);
 # None = not captured for the current kernels.
-NCU_TRAFFIC_PER_STEP = {"wht_project_mma_kernel": 867.8e6, "lbp_products_kernel": 275.4e6}
+NCU_TRAFFIC_PER_STEP = {"wht_project_mma_kernel": 868.2e6, "lbp_products_pair_kernel": 283.3e6}
 
 
 # ------------------------------------------------------------------ clocks ----
@@ -369,8 +369,8 @@ def run_gpu(args):
             ach = prod_bytes / (prod_ms * 1e-3) / 1e9
             r_prod = {"bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"],
                       "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4)}
-        r_prod.update({"kernel": "lbp_products_kernel",
-                       "traffic": NCU_TRAFFIC_PER_STEP["lbp_products_kernel"],
+        r_prod.update({"kernel": "lbp_products_pair_kernel",
+                       "traffic": NCU_TRAFFIC_PER_STEP["lbp_products_pair_kernel"],
                        "algorithmic_bytes": int(prod_bytes), "algorithmic_flops": prod_flops,
                        "launches_per_step": len(layers), "peak_source": peaks["source"],
                        "share_of_step": round(prod_ms / all_ms, 4)})
