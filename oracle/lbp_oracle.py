@@ -179,6 +179,33 @@ def expand(t_hat, k: int, bases) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------
+# Low-heuristic-error selection (Sec. 3.2): profile the energy of every basis
+# response, keep the r strongest.
+# --------------------------------------------------------------------------
+def spectrum(t, k: int) -> np.ndarray:
+    """E[i, j] = sum over blocks and channels of t_hat[.., (i,j), ..]^2 with all
+    k^2 bases active (orthonormal coefficients, so sum(E) = ||t||^2 by Parseval).
+
+    t (B,H,W,C) -> E (k, k), i the sequency along H, j along W.
+    """
+    all_pairs = [(i, j) for i in range(k) for j in range(k)]
+    t_hat = project(t, k, all_pairs)                     # (B, H/k, W/k, k^2, C)
+    return np.sum(t_hat * t_hat, axis=(0, 1, 2, 4)).reshape(k, k)
+
+
+def select_lhe(energy, k: int, r: int):
+    """The r bases with the largest energy, strongest first.  The paper does not
+    say how equal energies are ordered; here the lower-frequency pair (the
+    PREFIX order key) wins a tie, which makes the list unique."""
+    energy = np.asarray(energy, dtype=np.float64).reshape(k, k)
+    if not (1 <= r <= k * k):
+        raise ValueError("rank out of range")
+    pairs = [(i, j) for i in range(k) for j in range(k)]
+    pairs.sort(key=lambda ij: (-energy[ij[0], ij[1]],) + _prefix_key(*ij))
+    return pairs[:r]
+
+
+# --------------------------------------------------------------------------
 # Backward passes
 # --------------------------------------------------------------------------
 def backward_exact(x, g_y, w):

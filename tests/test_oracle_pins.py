@@ -407,3 +407,88 @@ def test_flops_worked_example_from_paper():
     cx, cy, L, r = g["Cx"], g["Cy"], g["L"], g["r"]
     assert over / mf["vanilla"] == pytest.approx((2 * cx + cy) * L * r / (4 * cx * cy * L), rel=1e-12)
     assert over / mf["vanilla"] == pytest.approx((1 / cy + 1 / (2 * cx)) * r / 2, rel=1e-12)
+
+
+# ------------------------------------------- LHE selection (Sec. 3.2) ----
+@pytest.mark.parametrize("k", KS)
+def test_spectrum_preserves_energy(k):
+    # Parseval (Sec. 3.2): the orthonormal WHT keeps the signal energy, so the
+    # energies of all k^2 responses add up to ||t||^2.
+    rng = np.random.default_rng(5)
+    t = rng.standard_normal((2, 2 * k, k, 3))
+    E = O.spectrum(t, k)
+    assert E.shape == (k, k) and np.all(E >= 0)
+    assert abs(E.sum() - np.sum(t * t)) <= 1e-10 * np.sum(t * t)
+
+
+@pytest.mark.parametrize("k", KS)
+def test_spectrum_matches_pointwise_definition(k):
+    # brute force from the definition of a response: Python loops over the
+    # block, Walsh rows built here from their sign-change count
+    rng = np.random.default_rng(6)
+    t = rng.standard_normal((1, k, 2 * k, 2))
+    H = np.array([[(-1) ** bin(a & b).count("1") for b in range(k)] for a in range(k)])
+    wal = {int(np.sum(H[a, 1:] != H[a, :-1])): H[a] for a in range(k)}
+    E = np.zeros((k, k))
+    for bw in range(2):
+        for c in range(2):
+            for i in range(k):
+                for j in range(k):
+                    acc = 0.0
+                    for u in range(k):
+                        for v in range(k):
+                            acc += wal[i][u] * wal[j][v] * t[0, u, bw * k + v, c]
+                    E[i, j] += (acc / k) ** 2
+    assert np.allclose(O.spectrum(t, k), E, rtol=1e-12, atol=1e-12)
+
+
+def test_spectrum_of_a_single_basis_function_is_a_single_peak():
+    # a block equal to amplitude * B_{i,j} has all its energy in response (i, j):
+    # pins the index order (i along H, j along W) and the orientation
+    k, i, j = 8, 2, 5
+    amp = np.array([1.0, -3.0, 0.5])
+    blk = O.basis_2d(k, i, j).astype(np.float64)                  # k x k, rows = H axis
+    t = (blk[None, :, :, None] * amp[None, None, None, :])
+    E = O.spectrum(t, k)
+    expect = np.zeros((k, k))
+    expect[i, j] = k * k * np.sum(amp ** 2)                       # ||t||^2
+    assert np.allclose(E, expect, atol=1e-9)
+    # the transposed pattern peaks at (j, i)
+    E2 = O.spectrum(np.transpose(t, (0, 2, 1, 3)), k)
+    assert np.argmax(E2) == j * k + i
+
+
+def test_block_constant_tensor_has_only_dc_energy():
+    k = 4
+    rng = np.random.default_rng(8)
+    coarse = rng.standard_normal((2, 3, 2, 5))
+    t = np.repeat(np.repeat(coarse, k, axis=1), k, axis=2)
+    E = O.spectrum(t, k)
+    assert E[0, 0] > 0 and np.allclose(np.delete(E.ravel(), 0), 0.0, atol=1e-12)
+
+
+def test_lhe_selection_takes_the_strongest_and_breaks_ties_by_frequency():
+    k = 4
+    E = np.zeros((k, k))
+    E[3, 3], E[0, 2], E[2, 0], E[1, 1], E[0, 0] = 9.0, 5.0, 5.0, 5.0, 1.0
+    # three equal energies on the anti-diagonal i + j = 2: the balanced pair
+    # first, then the smaller row index (the PREFIX order key)
+    assert O.select_lhe(E, k, 5) == [(3, 3), (1, 1), (0, 2), (2, 0), (0, 0)]
+    assert O.select_lhe(E, k, 1) == [(3, 3)]
+    full = O.select_lhe(E, k, k * k)
+    assert sorted(full) == [(i, j) for i in range(k) for j in range(k)]
+    with pytest.raises(ValueError):
+        O.select_lhe(E, k, 0)
+
+
+def test_lhe_on_a_decaying_spectrum_equals_the_low_pass_set():
+    # energy that falls strictly with the PREFIX order key: the strongest r
+    # responses are exactly the PREFIX-r (for triangular r: LP_L1) set
+    k = 8
+    order = O.select_bases(k, O.RULE_PREFIX, k * k)
+    E = np.zeros((k, k))
+    for rank, (i, j) in enumerate(order):
+        E[i, j] = 2.0 ** (-rank)
+    for r in (1, 3, 8, 10, 21):
+        assert O.select_lhe(E, k, r) == order[:r]
+    assert set(O.select_lhe(E, k, 10)) == set(O.select_bases(k, O.RULE_L1, 4))
