@@ -97,6 +97,14 @@ int lbp_select_bases(int k, int rule, int param, lbp_basis* out, int cap, int* r
  * k*k*r int8, row-major.  Validates the list like every other call. */
 int lbp_basis_matrix(int k, const lbp_basis* set, int r, int8_t* P_out);
 
+/* Sec. 3.2, low-heuristic-error (LHE) selection: the r bases with the largest
+ * profiled energy, strongest first.  energy: host array of k*k doubles as
+ * written by lbp_spectrum (index i*k + j).  The paper does not order equal
+ * energies; the pair that comes first in the PREFIX order wins a tie, so the
+ * list is unique.  out: host array of at least r entries.  LBP_ERR_BASIS for
+ * r outside 1..k*k or an energy that is negative or not finite. */
+int lbp_select_lhe(const double* energy, int k, int r, lbp_basis* out);
+
 /* Table 1 closed forms, in FLOPs.  which: 0 vanilla BP 4 Cx Cy L, 1 projection
  * (Cx+Cy) L r, 2 low-rank products 4 Cx Cy r, 3 reverse projection Cx L r,
  * 4 = 1+2+3.  Returns a negative number for a bad `which`. */
@@ -123,6 +131,18 @@ size_t lbp_status_bytes(void);
 int lbp_project(const void* t, void* t_hat, int B, int H, int W, int C, int k,
                 const lbp_basis* set, int r, int dtype,
                 void* ws, size_t ws_bytes, void* stream);
+
+/* Sec. 3.2 (LHE profiling): energy of every basis response of t,
+ *   energy[i*k + j] = sum over blocks and channels of t_hat[.., (i,j), ..]^2
+ * with t_hat the coefficients of Eq. 6 for all k*k bases, so that the k*k
+ * energies add up to ||t||^2.  t (B,H,W,C) of `dtype`; energy: DEVICE array of
+ * k*k doubles, overwritten.  The coefficients are materialised in `dtype`
+ * (fp32 accumulation, one rounding) in the workspace and their squares summed
+ * in fp32 per row, in fp64 across rows.
+ * ws: >= lbp_spectrum_workspace_bytes(...); 0 from that call = invalid shape. */
+size_t lbp_spectrum_workspace_bytes(int B, int H, int W, int C, int k, int dtype);
+int lbp_spectrum(const void* t, double* energy, int B, int H, int W, int C, int k, int dtype,
+                 void* ws, size_t ws_bytes, void* stream);
 
 /* Eq. 7 per block:  t[b,bh*k+u,bw*k+v,c] = (1/k) sum_q wal_iq[u] wal_jq[v]
  *                                          t_hat[b,bh,bw,q,c].

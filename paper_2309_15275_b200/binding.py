@@ -66,6 +66,12 @@ def _lib() -> C.CDLL:
         lib.lbp_workspace_bytes.restype = sz
         lib.lbp_status_bytes.argtypes = []
         lib.lbp_status_bytes.restype = sz
+        lib.lbp_select_lhe.argtypes = [C.POINTER(C.c_double), i32, i32, C.POINTER(Basis)]
+        lib.lbp_select_lhe.restype = i32
+        lib.lbp_spectrum_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32]
+        lib.lbp_spectrum_workspace_bytes.restype = sz
+        lib.lbp_spectrum.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp, sz, vp]
+        lib.lbp_spectrum.restype = i32
         for name in ("lbp_project", "lbp_expand"):
             f = getattr(lib, name)
             f.argtypes = [vp, vp, i32, i32, i32, i32, i32, C.POINTER(Basis), i32, i32, vp, sz, vp]
@@ -95,7 +101,8 @@ def _lib() -> C.CDLL:
 EXPORTED = ("lbp_select_bases", "lbp_basis_matrix", "lbp_flops", "lbp_status_string",
             "lbp_last_cuda_error", "lbp_workspace_bytes", "lbp_status_bytes", "lbp_project",
             "lbp_expand", "lbp_backward", "lbp_backward_fullrank", "lbp_poll_status",
-            "lbp_backward_static", "lbp_launch_count", "lbp_set_phase_events", "lbp_phase_count", "lbp_phase_name")
+            "lbp_backward_static", "lbp_launch_count", "lbp_set_phase_events", "lbp_phase_count",
+            "lbp_phase_name", "lbp_select_lhe", "lbp_spectrum_workspace_bytes", "lbp_spectrum")
 
 
 def _check(status: int, where: str) -> None:
@@ -184,6 +191,38 @@ def lbp_project(t: torch.Tensor, k: int, bases, out: torch.Tensor | None = None,
     _check(_lib().lbp_project(_dev(t, "t"), _dev(out, "t_hat"), B, H, W, Cc, k, _bases(bases), r,
                               _dtype_code(t.dtype), _dev(ws, "ws"), ws.numel(), _stream()),
            "lbp_project")
+    return out
+
+
+def lbp_select_lhe(energy, k: int, r: int) -> List[Tuple[int, int]]:
+    """The r bases with the largest energy (k x k array as returned by lbp_spectrum)."""
+    flat = [float(v) for v in (energy.reshape(-1).tolist() if hasattr(energy, "reshape") else energy)]
+    if len(flat) != k * k:
+        raise ValueError("energy must hold k*k values")
+    buf = (C.c_double * (k * k))(*flat)
+    out = (Basis * max(r, 1))()
+    _check(_lib().lbp_select_lhe(buf, k, r, out), "lbp_select_lhe")
+    return [(out[q].i, out[q].j) for q in range(r)]
+
+
+def lbp_spectrum_workspace_bytes(B: int, H: int, W: int, Cc: int, k: int, dtype_code: int) -> int:
+    return int(_lib().lbp_spectrum_workspace_bytes(B, H, W, Cc, k, dtype_code))
+
+
+def lbp_spectrum(t: torch.Tensor, k: int, out: torch.Tensor | None = None,
+                 ws: torch.Tensor | None = None) -> torch.Tensor:
+    """t (B,H,W,C) -> energy (k, k) float64 on the device: sum of squares of every basis response."""
+    B, H, W, Cc = t.shape
+    if out is None:
+        out = torch.empty((k, k), dtype=torch.float64, device=t.device)
+    if ws is None:
+        n = lbp_spectrum_workspace_bytes(B, H, W, Cc, k, _dtype_code(t.dtype))
+        if n == 0:
+            raise ValueError("invalid shape for lbp_spectrum_workspace_bytes")
+        ws = torch.empty(n, dtype=torch.uint8, device=t.device)
+    _check(_lib().lbp_spectrum(_dev(t, "t"), _dev(out, "energy"), B, H, W, Cc, k,
+                               _dtype_code(t.dtype), _dev(ws, "ws"), ws.numel(), _stream()),
+           "lbp_spectrum")
     return out
 
 

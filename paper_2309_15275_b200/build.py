@@ -12,7 +12,8 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblbp.so")
 
 SOURCES = ["lbp_host.cpp", "lbp_api.cu", "wht_project.cu", "wht_project_mma.cu", "wht_expand.cu",
-           "gemm_fp32.cu", "gemm_bf16.cu", "lbp_fused.cu", "lbp_fused2.cu", "lbp_static.cu"]
+           "gemm_fp32.cu", "gemm_bf16.cu", "lbp_fused.cu", "lbp_fused2.cu", "lbp_static.cu",
+           "wht_spectrum.cu"]
 
 
 def _nvcc() -> str:

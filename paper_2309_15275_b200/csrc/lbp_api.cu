@@ -210,6 +210,38 @@ int lbp_project(const void* t, void* t_hat, int B, int H, int W, int C, int k,
                         static_cast<uint32_t*>(ws), static_cast<cudaStream_t>(stream));
 }
 
+size_t lbp_spectrum_workspace_bytes(int B, int H, int W, int C, int k, int dtype) {
+  if (check_grid(B, H, W, C, k, dtype) != LBP_OK) return 0;
+  const size_t es = dtype == LBP_BF16 ? 2 : 4;
+  const size_t coef = static_cast<size_t>(B) * H * W * C * es;   // all k*k coefficients per block
+  return kStatusBytes + (coef + 255) / 256 * 256;
+}
+
+int lbp_spectrum(const void* t, double* energy, int B, int H, int W, int C, int k, int dtype,
+                 void* ws, size_t ws_bytes, void* stream) {
+  if (t == nullptr || energy == nullptr) return LBP_ERR_NULL;
+  if (int e = check_grid(B, H, W, C, k, dtype)) return e;
+  const int r = k * k;
+  lbp_basis all[256];
+  for (int i = 0; i < k; ++i)
+    for (int j = 0; j < k; ++j) all[i * k + j] = lbp_basis{i, j};
+  BasisPlan plan;
+  if (int e = make_basis_plan(k, all, r, &plan)) return e;
+  if (!aligned16(t) || !aligned16(ws) || (reinterpret_cast<uintptr_t>(energy) & 7u) != 0)
+    return LBP_ERR_ALIGN;
+  if (ws == nullptr || ws_bytes < lbp_spectrum_workspace_bytes(B, H, W, C, k, dtype))
+    return LBP_ERR_WORKSPACE;
+  if (int e = check_device_arch()) return e;
+  uint8_t* wsb = static_cast<uint8_t*>(ws);
+  void* coef = wsb + kStatusBytes;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (int e = launch_project(t, coef, dtype, B, H, W, C, plan, RowMap{1, r},
+                             static_cast<uint32_t*>(ws), st))
+    return e;
+  const long long rows = static_cast<long long>(B) * H * W;   // blocks * k * k
+  return launch_square_reduce(coef, dtype, rows, C, r, energy, st);
+}
+
 int lbp_expand(const void* t_hat, void* t, int B, int H, int W, int C, int k,
                const lbp_basis* set, int r, int dtype, void* ws, size_t ws_bytes, void* stream) {
   if (t == nullptr || t_hat == nullptr) return LBP_ERR_NULL;

@@ -3,6 +3,7 @@
 // plan the transform kernels consume.
 #include <algorithm>
 #include <cstring>
+#include <cmath>
 #include <vector>
 
 #include "lbp_internal.h"
@@ -126,6 +127,28 @@ int lbp_select_bases(int k, int rule, int param, lbp_basis* out, int cap, int* r
   for (size_t q = 0; q < sel.size(); ++q) {
     out[q].i = sel[q].i;
     out[q].j = sel[q].j;
+  }
+  return LBP_OK;
+}
+
+int lbp_select_lhe(const double* energy, int k, int r, lbp_basis* out) {
+  if (int e = check_order(k)) return e;
+  if (energy == nullptr || out == nullptr) return LBP_ERR_NULL;
+  if (r < 1 || r > k * k) return LBP_ERR_BASIS;
+  for (int n = 0; n < k * k; ++n)
+    if (!(energy[n] >= 0.0) || !std::isfinite(energy[n])) return LBP_ERR_BASIS;
+  std::vector<PairKey> all;
+  for (int i = 0; i < k; ++i)
+    for (int j = 0; j < k; ++j) all.push_back({i, j});
+  // strongest first; equal energies in the PREFIX order
+  std::sort(all.begin(), all.end(), [&](const PairKey& a, const PairKey& b) {
+    const double ea = energy[a.i * k + a.j], eb = energy[b.i * k + b.j];
+    if (ea != eb) return ea > eb;
+    return prefix_less(a, b);
+  });
+  for (int q = 0; q < r; ++q) {
+    out[q].i = all[q].i;
+    out[q].j = all[q].j;
   }
   return LBP_OK;
 }

@@ -88,6 +88,11 @@ int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* ou
                     int dtype, int B, int H, int W, const BasisPlan& plan, RowMap rows,
                     uint32_t* status, cudaStream_t stream);
 
+// energy[q] (device, r doubles, overwritten) = sum of squares of the rows
+// q, q + r, ... of t_hat (rows x C of `dtype`).
+int launch_square_reduce(const void* t_hat, int dtype, long long rows, int C, int r, double* energy,
+                         cudaStream_t stream);
+
 // t_hat is fp32 when `in_f32`, else of `dtype`; t is of `dtype`.
 int launch_expand(const void* t_hat, bool in_f32, void* t, int dtype, int B, int H, int W, int C,
                   const BasisPlan& plan, RowMap rows, cudaStream_t stream);

@@ -239,3 +239,71 @@ def test_repeated_calls_are_deterministic(dev):
     a = lbp.lbp_backward(xd, gd, wd, 8, bases)
     b = lbp.lbp_backward(xd, gd, wd, 8, bases)
     assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+# ------------------------------------------ LHE profiling (Sec. 3.2) ----
+def _low_frequency_tensor(shape, k, dtype, key):
+    """Noise plus a strong block-smooth part: most energy in the low responses,
+    as the paper reports for real gradients (Sec. 4, spectrum figure)."""
+    B, H, W, C = shape
+    fine = synth.make_tensor(shape, ("normal", 0.25), "f32", case_key=key)
+    coarse = synth.make_tensor((B, H // 2, W // 2, C), ("normal", 1.0), "f32", case_key=key + 1)
+    smooth = coarse.repeat_interleave(2, dim=1).repeat_interleave(2, dim=2)
+    return (fine + smooth).to(dtype)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("k", [4, 8, 16])
+def test_spectrum_matches_oracle(dev, dtype, k):
+    shape = (3, 2 * k, 3 * k, 200)   # several blocks, ragged channel tail
+    t = _low_frequency_tensor(shape, k, dtype, 900 + k)
+    e = lbp.lbp_spectrum(t.to(dev), k)
+    want = O.spectrum(f64(t), k)
+    got = e.cpu().numpy()
+    assert got.shape == (k, k)
+    # energies are sums of squares of coefficients held in `dtype`
+    tol = 1e-5 if dtype == torch.float32 else 2e-2
+    assert np.max(np.abs(got - want) / want.max()) <= tol
+    assert abs(got.sum() - np.sum(f64(t) ** 2)) <= tol * np.sum(f64(t) ** 2)   # Parseval
+    # the selection is taken on the host from the energies: same list wherever
+    # the oracle's energies are separated by more than the tolerance
+    for r in (1, 4, k):
+        sel = lbp.lbp_select_lhe(got, k, r)
+        ref = O.select_lhe(want, k, r)
+        srt = np.sort(want.ravel())[::-1]
+        if r < k * k and (srt[r - 1] - srt[r]) > 4 * tol * want.max():
+            assert set(sel) == set(ref)
+        assert sel == O.select_lhe(got, k, r)
+    # second call into the same output: overwritten, not accumulated
+    e2 = lbp.lbp_spectrum(t.to(dev), k, out=e)
+    assert np.allclose(e2.cpu().numpy(), got, rtol=1e-12)
+
+
+def test_spectrum_full_size_layer_and_lhe_backward(dev):
+    # g_y of the ViT-B qkv layer at full size; then Algorithm 1 on the selected bases
+    case = synth.config_cases(3)[0]
+    x, gy, w = _inputs(3, 0, None)
+    k = case.k
+    e = lbp.lbp_spectrum(gy.to(dev), k).cpu().numpy()
+    total = float(torch.sum(gy.to(dev).double() ** 2))
+    assert abs(e.sum() - total) <= 2e-2 * total
+    # sampled check against the oracle: 8 images
+    want = O.spectrum(f64(gy[:8]), k)
+    got8 = lbp.lbp_spectrum(gy[:8].contiguous().to(dev), k).cpu().numpy()
+    assert np.max(np.abs(got8 - want)) <= 2e-2 * want.max()
+    bases = lbp.lbp_select_lhe(e, k, 8)
+    assert len(set(bases)) == 8
+    xs, gs = x[:4].contiguous(), gy[:4].contiguous()
+    g_x, g_W = lbp.lbp_backward(xs.to(dev), gs.to(dev), w.to(dev), k, bases)
+    wx, ww = O.backward_lowrank(f64(xs), f64(gs), f64(w), k, bases)
+    assert rel(g_x, wx) <= 2e-2 and rel(g_W, ww) <= 2e-2
+
+
+def test_spectrum_argument_errors(dev):
+    t = torch.zeros((1, 8, 8, 64), dtype=torch.bfloat16, device=dev)
+    e = torch.full((8, 8), -1.0, dtype=torch.float64, device=dev)
+    with pytest.raises(lbp.LbpError) as err:
+        lbp.lbp_spectrum(t, 8, out=e, ws=torch.zeros(256, dtype=torch.uint8, device=dev))
+    assert err.value.status == 7 and float(e.min()) == -1.0
+    with pytest.raises(ValueError):
+        lbp.lbp_spectrum(torch.zeros((1, 8, 12, 64), dtype=torch.bfloat16, device=dev), 8)

@@ -88,3 +88,34 @@ def test_device_calls_fail_loudly_without_cuda_tensors():
     t = torch.zeros((1, 8, 8, 8), dtype=torch.float32)
     with pytest.raises(ValueError):
         lbp.lbp_project(t, 8, [(0, 0)], out=torch.zeros((1, 1, 1, 1, 8)), ws=torch.zeros(256, dtype=torch.uint8))
+
+
+@pytest.mark.parametrize("k", (4, 8, 16))
+def test_select_lhe_bit_exact_vs_oracle(k):
+    rng = np.random.default_rng(40 + k)
+    # distinct energies, then a quantised array with many ties
+    for energy in (rng.random((k, k)), np.round(rng.random((k, k)) * 4) / 4):
+        for r in (1, 2, k, k * k // 2, k * k):
+            assert lbp.lbp_select_lhe(energy, k, r) == O.select_lhe(energy, k, r)
+
+
+def test_select_lhe_argument_errors():
+    e = np.ones((8, 8))
+    for bad_r in (0, 65):
+        with pytest.raises(lbp.LbpError) as err:
+            lbp.lbp_select_lhe(e, 8, bad_r)
+        assert err.value.status == 4
+    bad = e.copy()
+    bad[1, 1] = -1.0
+    with pytest.raises(lbp.LbpError) as err:
+        lbp.lbp_select_lhe(bad, 8, 3)
+    assert err.value.status == 4
+    bad[1, 1] = float("nan")
+    with pytest.raises(lbp.LbpError) as err:
+        lbp.lbp_select_lhe(bad, 8, 3)
+    assert err.value.status == 4
+    with pytest.raises(lbp.LbpError) as err:
+        lbp.lbp_select_lhe(np.ones((5, 5)), 5, 3)
+    assert err.value.status == 3
+    assert lbp.lbp_spectrum_workspace_bytes(2, 16, 16, 64, 8, lbp.LBP_BF16) >= 2 * 16 * 16 * 64 * 2
+    assert lbp.lbp_spectrum_workspace_bytes(2, 15, 16, 64, 8, lbp.LBP_BF16) == 0
