@@ -235,6 +235,8 @@ int lbp_spectrum(const void* t, double* energy, int B, int H, int W, int C, int 
   uint8_t* wsb = static_cast<uint8_t*>(ws);
   void* coef = wsb + kStatusBytes;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (spectrum_mma_supported(k, dtype))   // one pass, nothing materialised
+    return launch_spectrum_mma(t, B, H, W, C, plan, energy, static_cast<uint32_t*>(ws), st);
   if (int e = launch_project(t, coef, dtype, B, H, W, C, plan, RowMap{1, r},
                              static_cast<uint32_t*>(ws), st))
     return e;

@@ -88,6 +88,12 @@ int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* ou
                     int dtype, int B, int H, int W, const BasisPlan& plan, RowMap rows,
                     uint32_t* status, cudaStream_t stream);
 
+// One-pass spectrum (bf16 data, k = 4 or 8): energy[i*k + j] of all k*k responses.
+// plan: all k*k pairs in raster order.
+bool spectrum_mma_supported(int k, int dtype);
+int launch_spectrum_mma(const void* t, int B, int H, int W, int C, const BasisPlan& plan,
+                        double* energy, uint32_t* status, cudaStream_t stream);
+
 // energy[q] (device, r doubles, overwritten) = sum of squares of the rows
 // q, q + r, ... of t_hat (rows x C of `dtype`).
 int launch_square_reduce(const void* t_hat, int dtype, long long rows, int C, int r, double* energy,
