@@ -312,6 +312,29 @@ def run_gpu(args):
             full_us = a.elapsed_time(b) * 1e3 / 5
             layer_rows[li]["fullrank_us"] = round(full_us, 2)
             layer_rows[li]["speedup_vs_fullrank"] = round(full_us / layer_rows[li]["us"], 3)
+    # ---- LHE profiling pass (Sec. 3.2) on g_y of every layer, outside the timed region ----
+    lhe_rows = []
+    if rank == 0:
+        for L in layers:
+            gy = L["gy"]
+            Bq, Hq, Wq, Cq = gy.shape
+            sws = torch.empty(lbp.lbp_spectrum_workspace_bytes(Bq, Hq, Wq, Cq, k, lbp.LBP_BF16),
+                              dtype=torch.uint8, device=dev)
+            e_out = torch.empty((k, k), dtype=torch.float64, device=dev)
+            for _ in range(2):
+                lbp.lbp_spectrum(gy, k, out=e_out, ws=sws)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(5):
+                lbp.lbp_spectrum(gy, k, out=e_out, ws=sws)
+            b.record()
+            torch.cuda.synchronize()
+            us = a.elapsed_time(b) * 1e3 / 5
+            nbytes = gy.numel() * gy.element_size()
+            lhe_rows.append({"layer": L["case"].name, "us": round(us, 2), "bytes": nbytes,
+                             "gbs": round(nbytes / us / 1e3, 1),
+                             "frac_of_hbm_peak": round(nbytes / us / 1e3 / peaks["hbm_gbs"], 4)})
+            del sws
     barrier()
 
     # ---- end to end: host buffers, copies inside the timed region ----
@@ -398,6 +421,7 @@ def run_gpu(args):
                                       "figures come from the steps that carry phase events, which "
                                       "cost about 2.5 us per event"},
             "layers": layer_rows,
+            "lhe_spectrum": lhe_rows,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps},
             "gpu_launches": int(launches),
