@@ -312,6 +312,39 @@ def run_gpu(args):
             full_us = a.elapsed_time(b) * 1e3 / 5
             layer_rows[li]["fullrank_us"] = round(full_us, 2)
             layer_rows[li]["speedup_vs_fullrank"] = round(full_us / layer_rows[li]["us"], 3)
+    # ---- the other ranks of the configuration (r = 2, 4, 16), outside the timed region ----
+    rank_rows = []
+    if rank == 0:
+        full_step_us = sum(r_["fullrank_us"] for r_ in layer_rows)
+        for rr in (2, 4, 8, 16):
+            bases_r = lbp.lbp_select_bases(k, lbp.SEL_PREFIX, rr)
+            wss = [lbp.alloc_workspace(L["x"], L["gy"], k, rr) for L in layers]
+
+            def one_step():
+                for L, w_ in zip(layers, wss):
+                    lbp.lbp_backward(L["x"], L["gy"], L["w"], k, bases_r, g_x=L["gx"], g_W=L["gw"], ws=w_)
+            for _ in range(3):
+                one_step()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(10):
+                one_step()
+            b.record()
+            torch.cuda.synchronize()
+            us = a.elapsed_time(b) * 1e3 / 10
+            roof = 0.0
+            for L in layers:
+                c = L["case"]
+                ab = 2 * c.tokens * (2 * c.Cin + c.Cout) + 2 * c.Cin * c.Cout + 4 * c.Cin * c.Cout
+                af = 4.0 * c.Cin * c.Cout * c.blocks * rr
+                roof += max(ab / (peaks["hbm_gbs"] * 1e9), af / (peaks["bf16_tflops"] * 1e12)) * 1e6
+            rank_rows.append({"r": rr, "us_per_step": round(us, 2),
+                              "tokens_per_s": tokens_per_step / (us * 1e-6),
+                              "roofline_us": round(roof, 2), "roofline_frac": round(roof / us, 4),
+                              "speedup_vs_fullrank": round(full_step_us / us, 3)})
+            del wss
+    barrier()
+
     # ---- LHE profiling pass (Sec. 3.2) on g_y of every layer, outside the timed region ----
     lhe_rows = []
     if rank == 0:
@@ -421,6 +454,7 @@ def run_gpu(args):
                                       "figures come from the steps that carry phase events, which "
                                       "cost about 2.5 us per event"},
             "layers": layer_rows,
+            "rank_sweep": rank_rows,
             "lhe_spectrum": lhe_rows,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps},

@@ -11,3 +11,4 @@ from .binding import (  # noqa: F401
     lbp_set_phase_events, lbp_backward_static, STATIC_SCRATCH_BYTES,
     lbp_select_lhe, lbp_spectrum, lbp_spectrum_workspace_bytes,
 )
+from .autograd import LbpLinear, LbpLinearFunction  # noqa: F401,E402

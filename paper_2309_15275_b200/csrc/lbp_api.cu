@@ -17,7 +17,17 @@ static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 int check_device_arch() {
   int dev = 0, major = 0;
+  // Every device entry point passes through here before it launches anything.
+  // A non-sticky error left behind on this thread by other code in the process
+  // (cudaGetLastError() not yet called on it) would otherwise be reported by
+  // the launch checks below as this library's own.
+  (void)cudaGetLastError();
   LBP_CUDA_TRY(cudaGetDevice(&dev));
+  // Tensor maps are encoded through the driver API, which needs the device's
+  // primary context current on the calling thread.  A thread that has made no
+  // runtime call yet (a framework's worker thread) has none: selecting the
+  // device it already has binds it, and changes nothing else.
+  LBP_CUDA_TRY(cudaSetDevice(dev));
   LBP_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
   return major == 10 ? LBP_OK : LBP_ERR_ARCH;
 }
@@ -65,7 +75,9 @@ int encode_block_tensor_map(CUtensorMap* map, const void* base, int dtype, int B
           CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
-    set_last_cuda_error(cudaErrorInvalidValue);
+    // CUresult and cudaError_t share their numbering
+    set_last_cuda_error(static_cast<cudaError_t>(r));
+    note_cuda_failure(static_cast<cudaError_t>(r), __FILE__, __LINE__);
     return LBP_ERR_CUDA;
   }
   return LBP_OK;
@@ -84,7 +96,9 @@ int encode_matrix_tensor_map(CUtensorMap* map, const void* base, long long rows,
                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
-    set_last_cuda_error(cudaErrorInvalidValue);
+    // CUresult and cudaError_t share their numbering
+    set_last_cuda_error(static_cast<cudaError_t>(r));
+    note_cuda_failure(static_cast<cudaError_t>(r), __FILE__, __LINE__);
     return LBP_ERR_CUDA;
   }
   return LBP_OK;

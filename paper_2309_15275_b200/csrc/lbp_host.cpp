@@ -2,6 +2,8 @@
 // matrix of Eq. 6, the cost model of Table 1, status strings, and the basis
 // plan the transform kernels consume.
 #include <algorithm>
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <cmath>
 #include <vector>
@@ -12,6 +14,11 @@ namespace lbp {
 
 static thread_local int g_last_cuda_error = 0;
 void set_last_cuda_error(cudaError_t e) { g_last_cuda_error = static_cast<int>(e); }
+void note_cuda_failure(cudaError_t e, const char* file, int line) {
+  const char* v = std::getenv("LBP_VERBOSE_ERRORS");
+  if (v != nullptr && v[0] == '1')
+    std::fprintf(stderr, "lbp: CUDA error %d at %s:%d\n", static_cast<int>(e), file, line);
+}
 
 thread_local long long g_launches = 0;
 void count_launch(int n) { g_launches += n; }

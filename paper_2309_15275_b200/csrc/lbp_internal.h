@@ -53,13 +53,15 @@ int check_order(int k);
 
 void set_last_cuda_error(cudaError_t e);
 void count_launch(int n = 1);   // bumps the per-thread kernel-launch counter
-#define LBP_CUDA_TRY(expr)                       \
-  do {                                           \
-    cudaError_t e__ = (expr);                    \
-    if (e__ != cudaSuccess) {                    \
-      ::lbp::set_last_cuda_error(e__);           \
-      return LBP_ERR_CUDA;                       \
-    }                                            \
+void note_cuda_failure(cudaError_t e, const char* file, int line);   // LBP_VERBOSE_ERRORS=1: one line on stderr
+#define LBP_CUDA_TRY(expr)                                 \
+  do {                                                     \
+    cudaError_t e__ = (expr);                              \
+    if (e__ != cudaSuccess) {                              \
+      ::lbp::set_last_cuda_error(e__);                     \
+      ::lbp::note_cuda_failure(e__, __FILE__, __LINE__);   \
+      return LBP_ERR_CUDA;                                 \
+    }                                                      \
   } while (0)
 
 // ---- tensor maps (TMA descriptors), encoded on the host ------------------

@@ -307,3 +307,24 @@ def test_spectrum_argument_errors(dev):
     assert err.value.status == 7 and float(e.min()) == -1.0
     with pytest.raises(ValueError):
         lbp.lbp_spectrum(torch.zeros((1, 8, 12, 64), dtype=torch.bfloat16, device=dev), 8)
+
+
+# ------------------------------------------------ autograd front end ----
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_autograd_linear_backward_is_algorithm_1(dev, dtype):
+    k, Cin, Cout = 8, 64, 96
+    name = "f32" if dtype == torch.float32 else "bf16"
+    x = synth.make_tensor((2, 16, 8, Cin), ("normal", 1.0), name, case_key=950)
+    gy = synth.make_tensor((2, 16, 8, Cout), ("normal", 1.0), name, case_key=951)
+    bases = O.select_bases(k, O.RULE_L1, 3)
+    layer = lbp.LbpLinear(Cin, Cout, k, bases, device=dev, dtype=dtype)
+    w = layer.weight.detach().clone()
+    xd = x.to(dev).requires_grad_(True)
+    y = layer(xd)
+    want_y = f64(x) @ f64(w).T
+    assert rel(y.detach(), want_y) <= TOL[dtype]
+    y.backward(gy.to(dev))
+    wx, ww = O.backward_lowrank(f64(x), f64(gy), f64(w), k, bases)
+    assert rel(xd.grad, wx) <= TOL[dtype]
+    assert rel(layer.weight.grad, ww) <= TOL[dtype]
+    assert layer.weight.grad.dtype == dtype
