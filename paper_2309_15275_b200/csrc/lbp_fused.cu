@@ -119,7 +119,7 @@ __device__ __forceinline__ Tile nth_tile(const FusedParams& p, int cta, int grid
 }
 
 // ------------------------------------------------------------------ kernel ----
-template <int K, int LB>
+template <int K, int LB, int NEX = 0>
 __global__ void __launch_bounds__(kThreads, 1)
     lbp_products_kernel(const __grid_constant__ CUtensorMap tm_gyhat_k,
                         const __grid_constant__ CUtensorMap tm_gyhat_mn,
@@ -289,7 +289,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       dt.slice = tl.slice;
       dt.tmem_acc = tmem_base + acc_col;
       uint64_t* release_bar = &acc_empty[slot];
-      drain_tile<K, LB>(p, fb, dt, Eg, bar_id, eg, etid, quarter, lane,
+      drain_tile<K, LB, NEX>(p, fb, dt, Eg, bar_id, eg, etid, quarter, lane,
                         [release_bar]() { ptx::mbar_arrive(release_bar); });
     }
     if (etid == 0) trace_mark(p, 4);   // latest of the groups
@@ -381,8 +381,38 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
   p.num_kb_w = p.G * (BM / BK);
   FusedBasis fb;
   for (int n = 0; n < 64; ++n) fb.qmap[n] = -1;
-  for (int a = 0; a < bp.LB; ++a)
-    for (int b = 0; b < bp.LB; ++b) fb.qmap[a * bp.LB + b] = bp.qmap[a * bp.LB + b];
+  for (int x = 0; x < kFusedMaxExtra; ++x) {
+    fb.ex_q[x] = -1;
+    fb.ex_mu[x] = fb.ex_mv[x] = 0;
+  }
+  p.lb_kernel = bp.LB;
+  p.n_extra = 0;
+  int n_outside = 0;   // bases with an index of 4 or more
+  for (int q = 0; q < bp.r; ++q) n_outside += (bp.seq_i[q] >= 4 || bp.seq_j[q] >= 4) ? 1 : 0;
+  if (bp.LB == 8 && n_outside <= kFusedMaxExtra) {
+    // An 8 x 8 coefficient array that is empty but for a few entries outside its
+    // 4 x 4 corner (PREFIX sets of rank 14-16): butterfly on the corner, the few
+    // others added token by token.
+    p.lb_kernel = 4;
+    int x = 0;
+    for (int q = 0; q < bp.r; ++q) {
+      if (bp.seq_i[q] < 4 && bp.seq_j[q] < 4) {
+        fb.qmap[walsh_natural_index(4, bp.seq_i[q]) * 4 + walsh_natural_index(4, bp.seq_j[q])] =
+            static_cast<int16_t>(q);
+      } else {
+        fb.ex_q[x] = static_cast<int16_t>(q);
+        for (int t = 0; t < K; ++t) {
+          if (__builtin_popcount(static_cast<unsigned>(bp.nat_i[q] & t)) & 1) fb.ex_mu[x] |= static_cast<uint16_t>(1u << t);
+          if (__builtin_popcount(static_cast<unsigned>(bp.nat_j[q] & t)) & 1) fb.ex_mv[x] |= static_cast<uint16_t>(1u << t);
+        }
+        ++x;
+      }
+    }
+    p.n_extra = x;
+  } else {
+    for (int a = 0; a < bp.LB; ++a)
+      for (int b = 0; b < bp.LB; ++b) fb.qmap[a * bp.LB + b] = bp.qmap[a * bp.LB + b];
+  }
   if (fused_pair_supported(L, sms))
     return launch_fused_pair(x, g_y, W, g_W, L, bp, p, fb, lay, sms, status, stream, hook, hook_arg);
 
@@ -534,7 +564,12 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
                                   p.gw_splits, p.gw_bf16 != 0, stream);
     return LBP_OK;
   };
-  switch (K * 100 + bp.LB) {
+  if (p.n_extra > 0) {
+    if (K == 8) return launch(lbp_products_kernel<8, 4, kFusedMaxExtra>);
+    if (K == 16) return launch(lbp_products_kernel<16, 4, kFusedMaxExtra>);
+    return LBP_ERR_BASIS;
+  }
+  switch (K * 100 + p.lb_kernel) {
     case 401: return launch(lbp_products_kernel<4, 1>);
     case 402: return launch(lbp_products_kernel<4, 2>);
     case 404: return launch(lbp_products_kernel<4, 4>);

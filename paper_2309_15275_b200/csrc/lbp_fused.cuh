@@ -22,6 +22,7 @@ struct FusedParams {
   int32_t gw_splits, kb_per_split_w;      // K slices of a GW tile (fp32 planes, reduced afterwards)
   float* gw_planes;                       // [gw_splits][Cout][Cin] when gw_splits > 1
   int32_t gw_bf16;
+  int32_t lb_kernel, n_extra;             // epilogue core size and bases added token by token (host dispatch)
   float scale;                            // 1/k
   __nv_bfloat16* x_hat;
   __nv_bfloat16* gy_hat;
@@ -31,8 +32,16 @@ struct FusedParams {
   unsigned long long* trace;              // optional role timeline, 8 slots per CTA (null = off)
 };
 
+constexpr int kFusedMaxExtra = 2;
+
 struct FusedBasis {
   int16_t qmap[64];   // natural-order LB x LB position -> basis slot, -1 unused
+  // Bases outside the LB x LB core (kernels instantiated with extras only): the
+  // epilogue adds them token by token.  ex_q: slot, -1 = none; bit u of ex_mu /
+  // bit v of ex_mv is set where the Walsh row along H / W is -1.
+  int16_t ex_q[kFusedMaxExtra];
+  uint16_t ex_mu[kFusedMaxExtra];
+  uint16_t ex_mv[kFusedMaxExtra];
 };
 
 constexpr size_t kFusedTraceBytes = 256 * 8 * 8;   // last bytes of the scratch region

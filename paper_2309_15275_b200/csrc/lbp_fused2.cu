@@ -36,6 +36,7 @@ namespace fused2 {
 
 using fused::BM;
 using fused::kEBytes;
+constexpr int fused_max_extra = kFusedMaxExtra;
 using fused::kEGroups;
 using fused::kEStride;
 
@@ -180,7 +181,7 @@ __device__ __forceinline__ PairTile nth_pair_tile(const FusedParams& p, int pair
 }
 
 // ------------------------------------------------------------------ kernel ----
-template <int K, int LB>
+template <int K, int LB, int NEX = 0>
 __global__ void __launch_bounds__(kThreads, 1)
     lbp_products_pair_kernel(const __grid_constant__ CUtensorMap tm_gyhat_k,
                              const __grid_constant__ CUtensorMap tm_gyhat_mn,
@@ -348,7 +349,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       dt.slice = tl.slice;
       dt.tmem_acc = tmem_base + slot * kSlotCols;
       const uint32_t release_bar = map_to_rank(ptx::smem_u32(&acc_empty[slot]), 0);
-      fused::drain_tile<K, LB>(p, fb, dt, Eg, bar_id, eg, etid, quarter, lane,
+      fused::drain_tile<K, LB, NEX>(p, fb, dt, Eg, bar_id, eg, etid, quarter, lane,
                                [release_bar]() { mbar_arrive_cluster(release_bar); });
       if (etid == 0 && eg == 0) trace_mark(p, 5, true);
     }
@@ -519,7 +520,12 @@ int launch_fused_pair(const void* x, const void* g_y, const void* W, void* g_W, 
                                   p.gw_splits, p.gw_bf16 != 0, stream);
     return LBP_OK;
   };
-  switch (L.k * 100 + bp.LB) {
+  if (p.n_extra > 0) {
+    if (L.k == 8) return launch(lbp_products_pair_kernel<8, 4, fused_max_extra>);
+    if (L.k == 16) return launch(lbp_products_pair_kernel<16, 4, fused_max_extra>);
+    return LBP_ERR_BASIS;
+  }
+  switch (L.k * 100 + p.lb_kernel) {
     case 401: return launch(lbp_products_pair_kernel<4, 1>);
     case 402: return launch(lbp_products_pair_kernel<4, 2>);
     case 404: return launch(lbp_products_pair_kernel<4, 4>);

@@ -47,7 +47,7 @@ struct DrainTile {
 
 // `release()` is called by lane 0 of every warp once the warp has read its last
 // accumulator column (the tensor core may then overwrite the slot).
-template <int K, int LB, class Release>
+template <int K, int LB, int NEX, class Release>
 __device__ __forceinline__ void drain_tile(const FusedParams& p, const FusedBasis& fb,
                                            const DrainTile& t, float* Eg, int bar_id, int eg,
                                            int etid, int quarter, int lane, Release release) {
@@ -176,6 +176,59 @@ __device__ __forceinline__ void drain_tile(const FusedParams& p, const FusedBasi
           const int bw = blk % p.Wb, t2 = blk / p.Wb, bh = t2 % p.Hb, b = t2 / p.Hb;
           __nv_bfloat16* o = p.g_x +
                              ((static_cast<long long>(b) * p.H + bh * K) * p.W + bw * K) * p.Cin + ch;
+          if constexpr (NEX > 0) {
+            // Bases outside the LB x LB core: B_{i,j}[u][v] = s_i(u) s_j(v) with
+            // s = +-1, so each adds +-coefficient to every token.  The row sign is
+            // folded into the coefficient once per token row, the column sign is
+            // a +-1.0 factor of an FMA.
+            static_assert(NCH == 4, "extras go with four channels per thread");
+            float ce[NEX][NCH];
+            uint32_t mu[NEX], mv[NEX];
+#pragma unroll
+            for (int x = 0; x < NEX; ++x) {
+              const int q = fb.ex_q[x];
+              const int row_q = q >= 0 ? row_b + q : BM;
+              const float4 f =
+                  *reinterpret_cast<const float4*>(Eg + row_q * kEStride + ((cc ^ (row_q & 7)) << 2));
+              ce[x][0] = f.x;
+              ce[x][1] = f.y;
+              ce[x][2] = f.z;
+              ce[x][3] = f.w;
+              mu[x] = fb.ex_mu[x];
+              mv[x] = fb.ex_mv[x];
+            }
+#pragma unroll
+            for (int a = 0; a < LB; ++a) {
+#pragma unroll 1
+              for (int du = 0; du < RUN; ++du) {
+                const int u = a * RUN + du;
+                float ceu[NEX][NCH];
+#pragma unroll
+                for (int x = 0; x < NEX; ++x) {
+                  const float su = __uint_as_float(0x3f800000u | (((mu[x] >> u) & 1u) << 31));
+#pragma unroll
+                  for (int c = 0; c < NCH; ++c) ceu[x][c] = ce[x][c] * su;
+                }
+                __nv_bfloat16* orow = o + u * row_stride;
+#pragma unroll
+                for (int v = 0; v < K; ++v) {
+                  float val[NCH];
+#pragma unroll
+                  for (int c = 0; c < NCH; ++c) val[c] = acc[a][v / RUN][c];
+#pragma unroll
+                  for (int x = 0; x < NEX; ++x) {
+                    const float sv = __uint_as_float(0x3f800000u | ((mv[x] << (31 - v)) & 0x80000000u));
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) val[c] = fmaf(sv, ceu[x][c], val[c]);
+                  }
+                  uint2 pk;
+                  pk.x = pack_bf16x2(val[0] * p.scale, val[1] * p.scale);
+                  pk.y = pack_bf16x2(val[2] * p.scale, val[3] * p.scale);
+                  *reinterpret_cast<uint2*>(orow + v * tok_stride) = pk;
+                }
+              }
+            }
+          } else {
           // each of the LB x LB values covers a RUN x RUN patch of tokens: scale,
           // round and pack once, store RUN * RUN times
 #pragma unroll
@@ -209,6 +262,7 @@ __device__ __forceinline__ void drain_tile(const FusedParams& p, const FusedBasi
                                                  (b2 * RUN + dv) * tok_stride) = pk;
               }
             }
+          }
           }
         }
       }

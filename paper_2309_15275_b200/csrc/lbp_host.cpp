@@ -80,6 +80,8 @@ int make_basis_plan(int k, const lbp_basis* set, int r, BasisPlan* plan) {
     plan->qmap[a * LB + b] = static_cast<int16_t>(q);
     plan->nat_i[q] = static_cast<uint8_t>(walsh_natural_index(k, set[q].i));
     plan->nat_j[q] = static_cast<uint8_t>(walsh_natural_index(k, set[q].j));
+    plan->seq_i[q] = static_cast<uint8_t>(set[q].i);
+    plan->seq_j[q] = static_cast<uint8_t>(set[q].j);
   }
   return LBP_OK;
 }

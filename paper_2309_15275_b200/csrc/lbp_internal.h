@@ -39,6 +39,9 @@ struct BasisPlan {
   // wal_{i_q}[u] = (-1)^popcount(nat_i[q] & u), likewise for j along W
   uint8_t nat_i[kMaxRank];
   uint8_t nat_j[kMaxRank];
+  // the selected pairs themselves (sequency indices), slot by slot
+  uint8_t seq_i[kMaxRank];
+  uint8_t seq_j[kMaxRank];
 };
 
 // Validates (k, set, r) and fills `plan`.  Returns an lbp_status.
