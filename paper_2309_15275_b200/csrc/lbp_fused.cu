@@ -315,7 +315,15 @@ bool fused_supported(const lbp_layer& L, const BasisPlan& bp) {
 
 size_t fused_scratch_bytes(const lbp_layer& L, int r, FusedLayout* lay) {
   const long long nb = static_cast<long long>(L.B) * (L.H / L.k) * (L.W / L.k);
-  const int bpt = 128 / r;
+  // Blocks per 128-row group.  With very few groups (low rank on a small token
+  // grid) the expansion of a whole group, (128 / r) * k * k tokens per tile, falls
+  // on a handful of CTAs: groups are then filled only partly (rows left zero)
+  // until there are about two dozen 256-row tiles per column strip.
+  int bpt = 128 / r;
+  {
+    const long long n_tx = (L.Cin + 127) / 128;
+    while (bpt > 1 && ((nb + bpt - 1) / bpt + 1) / 2 * n_tx < 24) bpt = (bpt + 1) / 2;
+  }
   const long long G = (nb + bpt - 1) / bpt;
   FusedLayout l;
   size_t off = 0;

@@ -165,7 +165,7 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
       }
     }
     // rows of a padded row tile that no block owns are kept at zero
-    if (p.bpt > 1 && ((blk % p.bpt) == p.bpt - 1 || blk == p.nb - 1)) {
+    if ((blk % p.bpt) == p.bpt - 1 || blk == p.nb - 1) {
       const long long tile_base = static_cast<long long>(blk / p.bpt) * p.tile_rows;
       const int c = chunk * 64 + lane * 2;
       if (c < C)
