@@ -58,6 +58,11 @@ static int get_encode_fn(EncodeTiledFn* out) {
 
 int encode_block_tensor_map(CUtensorMap* map, const void* base, int dtype, int B, int H, int W,
                             int C, int k, int box_c, bool swizzle128) {
+  return encode_box_tensor_map(map, base, dtype, B, H, W, C, box_c, k, k, swizzle128);
+}
+
+int encode_box_tensor_map(CUtensorMap* map, const void* base, int dtype, int B, int H, int W, int C,
+                          int box_c, int box_w, int box_h, bool swizzle128) {
   EncodeTiledFn enc;
   if (int e = get_encode_fn(&enc)) return e;
   const cuuint64_t es = static_cast<cuuint64_t>(elem_size(dtype));
@@ -65,8 +70,8 @@ int encode_block_tensor_map(CUtensorMap* map, const void* base, int dtype, int B
                               static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(B)};
   const cuuint64_t strides[3] = {dims[0] * es, dims[0] * dims[1] * es,
                                  dims[0] * dims[1] * dims[2] * es};
-  const cuuint32_t box[4] = {static_cast<cuuint32_t>(box_c), static_cast<cuuint32_t>(k),
-                             static_cast<cuuint32_t>(k), 1u};
+  const cuuint32_t box[4] = {static_cast<cuuint32_t>(box_c), static_cast<cuuint32_t>(box_w),
+                             static_cast<cuuint32_t>(box_h), 1u};
   const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
   const CUresult r =
       enc(map, dtype == LBP_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,

@@ -72,6 +72,9 @@ void note_cuda_failure(cudaError_t e, const char* file, int line);   // LBP_VERB
 // channels; no swizzle, or the 128-byte swizzle (box_c * element size must be 128).
 int encode_block_tensor_map(CUtensorMap* map, const void* base, int dtype, int B, int H, int W,
                             int C, int k, int box_c, bool swizzle128);
+// Same tensor with an explicit box of box_h x box_w tokens.
+int encode_box_tensor_map(CUtensorMap* map, const void* base, int dtype, int B, int H, int W, int C,
+                          int box_c, int box_w, int box_h, bool swizzle128);
 // 2-D row-major bf16 matrix (rows, cols): box = box_rows x 64 columns (128 B),
 // 128-byte swizzle.
 int encode_matrix_tensor_map(CUtensorMap* map, const void* base, long long rows, long long cols,

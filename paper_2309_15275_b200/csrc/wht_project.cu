@@ -294,6 +294,19 @@ int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* ou
   if (dtype == LBP_BF16 && project_mma_supported(K, bp.r)) {
     // bf16 data at moderate rank: the +-1 basis matrix is applied on the tensor pipe
     CUtensorMap sw[2];
+    if (project_mma_strips(K, bp.r)) {
+      // order 4 works on strips of four blocks along W (4 x 16 token boxes)
+      if (int e = encode_box_tensor_map(&sw[0], t0, dtype, B, H, W, C0, box_c, 16, 4, true)) return e;
+      sw[1] = sw[0];
+      if (t1 != nullptr)
+        if (int e = encode_box_tensor_map(&sw[1], t1, dtype, B, H, W, C1, box_c, 16, 4, true)) return e;
+      ProjParams ps = p;
+      const long long strips = static_cast<long long>(B) * p.Hb * ((p.Wb + 3) / 4);
+      ps.n_items0 = static_cast<uint32_t>(strips * p.n_chunks[0]);
+      ps.n_items = ps.n_items0 + (t1 ? static_cast<uint32_t>(strips * p.n_chunks[1]) : 0u);
+      return launch_project_mma(sw, static_cast<__nv_bfloat16*>(out0),
+                                static_cast<__nv_bfloat16*>(out1), ps, bp, sms, stream);
+    }
     if (int e = encode_block_tensor_map(&sw[0], t0, dtype, B, H, W, C0, K, box_c, true)) return e;
     sw[1] = sw[0];
     if (t1 != nullptr)

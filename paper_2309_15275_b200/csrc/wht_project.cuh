@@ -30,6 +30,8 @@ struct ProjCfg {
 
 // Tensor-pipe projection (bf16 data): supported ranks per order.
 bool project_mma_supported(int k, int r);
+// Order 4 at low rank: items are strips of four blocks (4 x 16 token boxes).
+bool project_mma_strips(int k, int r);
 int launch_project_mma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloat16* out1,
                        const ProjParams& p, const BasisPlan& bp, int sms, cudaStream_t stream);
 

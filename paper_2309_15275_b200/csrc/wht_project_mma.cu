@@ -181,6 +181,176 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
   }
 }
 
+// Order 4: a block is only 16 tokens (2 KB per 64 channels), too little per
+// TMA request and per barrier wait.  One item is a strip of four blocks that are
+// neighbours along W: a 4 x 16 token box, 8 KB, the tile size of order 8.  Row
+// u * 16 + v of the tile holds token (u, v) of the strip; block j owns v = 4j..4j+3.
+constexpr int kStripBlocks = 4;
+constexpr int kStripWarps = 12, kStripStages = 2, kStripTileBytes = 64 * 128;
+constexpr int kStripSmemBytes =
+    kStripWarps * kStripStages * kStripTileBytes + kStripWarps * kStripStages * 8 + 1024;
+
+__global__ void __launch_bounds__(kStripWarps * 32, 1)
+    wht_project_mma_strip4_kernel(const __grid_constant__ CUtensorMap tmap0,
+                                  const __grid_constant__ CUtensorMap tmap1,
+                                  __nv_bfloat16* __restrict__ out0, __nv_bfloat16* __restrict__ out1,
+                                  const __grid_constant__ ProjParams p,
+                                  const __grid_constant__ MmaPlan mp) {
+  constexpr int K = 4, NW = kStripWarps, S = kStripStages;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + NW * S * kStripTileBytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, tq = lane & 3;
+  uint64_t* my_bars = bars + warp * S;
+  uint8_t* my_tiles = tiles + warp * S * kStripTileBytes;
+
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < S; ++s) ptx::mbar_init(&my_bars[s], 1);
+    ptx::mbar_fence_init();
+  }
+  if (threadIdx.x == 0) {
+    ptx::prefetch_tensormap(&tmap0);
+    ptx::prefetch_tensormap(&tmap1);
+  }
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  __syncthreads();
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // see wht_project_mma_kernel
+
+  // items count strips here: p.n_items0 / p.n_items = strips * chunks
+  const uint32_t first = blockIdx.x * NW + warp;
+  const uint32_t stride = gridDim.x * NW;
+  const uint32_t n_my = first < p.n_items ? (p.n_items - first + stride - 1) / stride : 0;
+  const uint32_t Wb4 = (static_cast<uint32_t>(p.Wb) + kStripBlocks - 1) / kStripBlocks;
+
+  auto issue = [&](uint32_t idx, int s) {
+    uint32_t item = first + idx * stride;
+    const int which = item >= p.n_items0;
+    if (which) item -= p.n_items0;
+    const uint32_t nch = static_cast<uint32_t>(p.n_chunks[which]);
+    const uint32_t sg = item / nch, chunk = item - sg * nch;
+    const uint32_t bw4 = sg % Wb4, t2 = sg / Wb4, bh = t2 % p.Hb, b = t2 / p.Hb;
+    ptx::mbar_expect_tx(&my_bars[s], static_cast<uint32_t>(kStripTileBytes));
+    // tokens past W (a last strip of fewer than four blocks) are zero-filled
+    ptx::tma_load_4d(my_tiles + s * kStripTileBytes, which ? &tmap1 : &tmap0, &my_bars[s],
+                     chunk * 64, bw4 * (K * kStripBlocks), bh * K, b);
+  };
+  if (lane == 0) {
+    for (uint32_t i = 0; i < S && i < n_my; ++i) issue(i, i);
+  }
+
+  uint32_t afrag[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int q = g + (j & 1) * 8;
+    const int tok = 2 * tq + (j >> 1) * 8;
+    afrag[j] = basis_bits<K>(mp, q, p.r, tok) | (basis_bits<K>(mp, q, p.r, tok + 1) << 16);
+  }
+
+  // token t = 4 u + dv of block j sits in tile row 16 u + 4 j + dv
+  const int ld_tok = ((lane >> 3) & 1) * 8 + (lane & 7);
+  const int ld_row0 = (ld_tok >> 2) * 16 + (ld_tok & 3);
+  const int ld_chunk = lane >> 4;
+
+  for (uint32_t idx = 0; idx < n_my; ++idx) {
+    const int s = static_cast<int>(idx % S);
+    const uint32_t parity = (idx / S) & 1u;
+    const bool ok = ptx::mbar_wait(&my_bars[s], parity, p.status, (3u << 16) | 2u);
+    if (!__all_sync(0xffffffffu, ok)) break;
+
+    uint32_t item = first + idx * stride;
+    const int which = item >= p.n_items0;
+    if (which) item -= p.n_items0;
+    const uint32_t nch = static_cast<uint32_t>(p.n_chunks[which]);
+    const uint32_t sg = item / nch;
+    const int chunk = static_cast<int>(item - sg * nch);
+    const uint32_t bw4 = sg % Wb4, t2 = sg / Wb4, bh = t2 % p.Hb, b = t2 / p.Hb;
+    const int C = p.C[which];
+    __nv_bfloat16* __restrict__ out = which ? out1 : out0;
+    const uint32_t tile = ptx::smem_u32(my_tiles + s * kStripTileBytes);
+    const int cbase = chunk * 64 + 2 * tq;
+
+#pragma unroll
+    for (int j = 0; j < kStripBlocks; ++j) {
+      const int bw = static_cast<int>(bw4) * kStripBlocks + j;
+      if (bw < p.Wb) {
+        const int blk = static_cast<int>((b * p.Hb + bh) * p.Wb) + bw;
+        float d[8][4];
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) d[nt][jj] = 0.f;
+        const int row = ld_row0 + 4 * j;
+#pragma unroll
+        for (int np = 0; np < 4; ++np) {
+          const int c16 = np * 2 + ld_chunk;
+          uint32_t b0, b1, b2, b3;
+          ldmatrix_x4_trans(tile + row * 128 + ((c16 ^ (row & 7)) << 4), b0, b1, b2, b3);
+          mma_bf16_16816(d[2 * np], afrag, b0, b1);
+          mma_bf16_16816(d[2 * np + 1], afrag, b2, b3);
+        }
+        const long long row0 = static_cast<long long>(blk / p.bpt) * p.tile_rows +
+                               static_cast<long long>(blk % p.bpt) * p.r;
+        const int q0 = g, q1 = g + 8;
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+          const int c = cbase + nt * 8;
+          if (c < C) {
+            if (q0 < p.r)
+              *reinterpret_cast<uint32_t*>(out + (row0 + q0) * C + c) =
+                  pack_bf16x2(d[nt][0] * p.scale, d[nt][1] * p.scale);
+            if (q1 < p.r)
+              *reinterpret_cast<uint32_t*>(out + (row0 + q1) * C + c) =
+                  pack_bf16x2(d[nt][2] * p.scale, d[nt][3] * p.scale);
+          }
+        }
+        // rows of a padded row tile that no block owns are kept at zero
+        if ((blk % p.bpt) == p.bpt - 1 || blk == p.nb - 1) {
+          const long long tile_base = static_cast<long long>(blk / p.bpt) * p.tile_rows;
+          const int c = chunk * 64 + lane * 2;
+          if (c < C)
+            for (long long r2 = row0 + p.r; r2 < tile_base + p.tile_rows; ++r2)
+              *reinterpret_cast<uint32_t*>(out + r2 * C + c) = 0u;
+        }
+      }
+    }
+
+    __syncwarp();
+    if (lane == 0 && idx + S < n_my) {
+      ptx::fence_proxy_async_smem();
+      issue(idx + S, s);
+    }
+  }
+}
+
+static int launch_strip4(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloat16* out1,
+                         const ProjParams& p, const MmaPlan& mp, int sms, cudaStream_t stream) {
+  auto kern = wht_project_mma_strip4_kernel;
+  LBP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kStripSmemBytes));
+  const uint32_t want = (p.n_items + kStripWarps - 1) / kStripWarps;
+  const int grid = static_cast<int>(want < static_cast<uint32_t>(sms) ? want : sms);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kStripWarps * 32);
+  cfg.dynamicSmemBytes = kStripSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  LBP_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmaps[0], tmaps[1], out0, out1, p, mp));
+  count_launch();
+  LBP_CUDA_TRY(cudaGetLastError());
+  return LBP_OK;
+}
+
+bool project_mma_strips(int k, int r) { return k == 4 && r <= 8; }
+
 bool project_mma_supported(int k, int r) {
   if (k == 4) return r <= 16;
   if (k == 8) return r <= 32;
@@ -228,7 +398,11 @@ int launch_project_mma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloa
   }
   const int mt = (bp.r + 15) / 16;
   switch (bp.k) {
-    case 4: return launch_mma_one<4, 1>(tmaps, out0, out1, p, mp, sms, stream);
+    case 4:
+      // few output rows: strips of four blocks (the caller encoded strip maps and
+      // counted strips); at higher rank the stores of a strip outlast its loads
+      if (project_mma_strips(bp.k, bp.r)) return launch_strip4(tmaps, out0, out1, p, mp, sms, stream);
+      return launch_mma_one<4, 1>(tmaps, out0, out1, p, mp, sms, stream);
     case 8:
       if (mt == 1) return launch_mma_one<8, 1>(tmaps, out0, out1, p, mp, sms, stream);
       return launch_mma_one<8, 2>(tmaps, out0, out1, p, mp, sms, stream);
