@@ -63,7 +63,7 @@ __device__ __forceinline__ void trace_mark(const FusedParams& p, int slot, bool 
 }
 
 // Tile list.  Tiles are numbered with the GW tiles (the larger ones) first and
-// dealt to the CTAs in a snake: round 0 forwards, round 1 backwards, ... so
+// dealt to the CTAs in a snake: first pass forwards, second pass backwards, ... so
 // that a CTA that got a large tile gets its next one last.  A CTA takes its
 // tiles in list order (walking the list backwards, GX tiles first, measured no
 // faster).
