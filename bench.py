@@ -375,22 +375,47 @@ def run_gpu(args):
     h2d = sum(L[n].numel() * L[n].element_size() for L in layers for n in ("x_h", "gy_h", "w_h"))
     d2h = sum(L[n].numel() * L[n].element_size() for L in layers for n in ("gx_h", "gw_h"))
 
+    # Copies run on two side streams so that the host-to-device copy of the next
+    # layer, the kernels of this layer and the device-to-host copy of the previous
+    # one overlap (PCIe is full duplex); events order every reuse of a buffer.
+    cur = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    for L in layers:
+        L["ev_in"], L["ev_done"], L["ev_out"] = (torch.cuda.Event() for _ in range(3))
+        L["ev_done"].record(cur)
+        L["ev_out"].record(cur)
+
     def e2e_step():
         for L in layers:
-            L["x"].copy_(L["x_h"], non_blocking=True)
-            L["gy"].copy_(L["gy_h"], non_blocking=True)
-            L["w"].copy_(L["w_h"], non_blocking=True)
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(L["ev_done"])          # the previous step's kernels read these buffers
+                L["x"].copy_(L["x_h"], non_blocking=True)
+                L["gy"].copy_(L["gy_h"], non_blocking=True)
+                L["w"].copy_(L["w_h"], non_blocking=True)
+                L["ev_in"].record(s_in)
+            cur.wait_event(L["ev_in"])
+            cur.wait_event(L["ev_out"])                # the previous step's results have left g_x / g_W
             lbp.lbp_backward(L["x"], L["gy"], L["w"], k, bases, g_x=L["gx"], g_W=L["gw"], ws=L["ws"])
             allreduce_gw(L["gw"])
-            L["gx_h"].copy_(L["gx"], non_blocking=True)
-            L["gw_h"].copy_(L["gw"], non_blocking=True)
+            L["ev_done"].record(cur)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(L["ev_done"])
+                L["gx_h"].copy_(L["gx"], non_blocking=True)
+                L["gw_h"].copy_(L["gw"], non_blocking=True)
+                L["ev_out"].record(s_out)
+
+    def e2e_join():
+        for L in layers:
+            cur.wait_event(L["ev_out"])
 
     e2e_step()
+    e2e_join()
     barrier()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record()
     for _ in range(e2e_steps):
         e2e_step()
+    e2e_join()                                         # every result is in host memory
     b.record()
     barrier()
     e2e_ms = a.elapsed_time(b) / e2e_steps
