@@ -208,15 +208,22 @@ def run_gpu(args):
     tokens_per_step = cases[0].tokens          # per GPU
 
     def step(record=None):
+        if record is None:
+            # the four layers are independent problems with their own buffers: one call
+            lbp.lbp_backward_batch([L["x"] for L in layers], [L["gy"] for L in layers],
+                                   [L["w"] for L in layers], k, bases,
+                                   g_xs=[L["gx"] for L in layers], g_Ws=[L["gw"] for L in layers],
+                                   wss=[L["ws"] for L in layers])
+            for L in layers:
+                allreduce_gw(L["gw"])   # data-parallel exchange; no-op on one GPU
+            return
         for li, L in enumerate(layers):
-            if record is not None:
-                # boundaries used: 0 start, 1 after the projection, 3 after the products kernel
-                lbp.lbp_set_phase_events([e if i in (0, 1, 3) else None
-                                          for i, e in enumerate(record[li])])
+            # boundaries used: 0 start, 1 after the projection, 3 after the products kernel
+            lbp.lbp_set_phase_events([e if i in (0, 1, 3) else None
+                                      for i, e in enumerate(record[li])])
             lbp.lbp_backward(L["x"], L["gy"], L["w"], k, bases, g_x=L["gx"], g_W=L["gw"], ws=L["ws"])
-            allreduce_gw(L["gw"])   # data-parallel exchange; no-op on one GPU
-        if record is not None:
-            lbp.lbp_set_phase_events(None)
+            allreduce_gw(L["gw"])
+        lbp.lbp_set_phase_events(None)
 
     def barrier():
         if world > 1:

@@ -60,7 +60,8 @@ typedef enum {
   LBP_ERR_ARCH = 8,       /* current device is not compute capability 10.x      */
   LBP_ERR_CUDA = 9,       /* a CUDA call failed; see lbp_last_cuda_error()      */
   LBP_ERR_TIMEOUT = 10,   /* a bounded device-side wait expired                 */
-  LBP_ERR_CAPACITY = 11   /* output array too small (lbp_select_bases)          */
+  LBP_ERR_CAPACITY = 11,  /* output array too small (lbp_select_bases)          */
+  LBP_ERR_OVERLAP = 12    /* buffers of different problems of a batch overlap   */
 } lbp_status;
 
 typedef enum { LBP_F32 = 0, LBP_BF16 = 1 } lbp_dtype;
@@ -163,6 +164,20 @@ int lbp_backward(const void* x, const void* g_y, const void* W,
                  void* g_x, void* g_W, const lbp_layer* layer,
                  const lbp_basis* set, int r,
                  void* ws, size_t ws_bytes, void* stream);
+
+/* Algorithm 1 for n (1..64) independent problems in one call, e.g. the linear
+ * layers of a block whose inputs are all at hand: problem i is
+ * lbp_backward(x[i], g_y[i], W[i], g_x[i], g_W[i], &layers[i], set, r, ws[i],
+ * ws_bytes[i]) and gives bit-identical results.  x .. ws, ws_bytes: host arrays
+ * of n entries.  What one problem writes (g_x, g_W, ws) no other problem may
+ * read or write (LBP_ERR_OVERLAP); inputs may be shared.  Knowing that, the
+ * library lets the projection kernel of problem i + 1 start on the SMs that the
+ * products kernel of problem i has already left instead of waiting for its last
+ * tile.  All arguments are checked before anything is enqueued. */
+int lbp_backward_batch(int n, const void* const* x, const void* const* g_y, const void* const* W,
+                       void* const* g_x, void* const* g_W, const lbp_layer* layers,
+                       const lbp_basis* set, int r, void* const* ws, const size_t* ws_bytes,
+                       void* stream);
 
 /* Eq. 2, exact backpropagation: g_W = g_y^T x over all tokens, g_x = g_y W.
  * This is what all k*k bases give (P P^T = I), computed without transforms.

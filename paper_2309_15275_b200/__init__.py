@@ -9,6 +9,6 @@ from .binding import (  # noqa: F401
     lbp_flops, lbp_poll_status, lbp_project, lbp_select_bases, lbp_status_bytes,
     lbp_status_string, lbp_workspace_bytes, lbp_launch_count, lbp_phase_count, lbp_phase_name,
     lbp_set_phase_events, lbp_backward_static, STATIC_SCRATCH_BYTES,
-    lbp_select_lhe, lbp_spectrum, lbp_spectrum_workspace_bytes,
+    lbp_select_lhe, lbp_spectrum, lbp_spectrum_workspace_bytes, lbp_backward_batch,
 )
 from .autograd import LbpLinear, LbpLinearFunction  # noqa: F401,E402

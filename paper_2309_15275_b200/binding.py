@@ -79,6 +79,10 @@ def _lib() -> C.CDLL:
         lib.lbp_backward.argtypes = [vp, vp, vp, vp, vp, C.POINTER(Layer), C.POINTER(Basis), i32,
                                      vp, sz, vp]
         lib.lbp_backward.restype = i32
+        lib.lbp_backward_batch.argtypes = [i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
+                                           C.POINTER(vp), C.POINTER(vp), C.POINTER(Layer),
+                                           C.POINTER(Basis), i32, C.POINTER(vp), C.POINTER(sz), vp]
+        lib.lbp_backward_batch.restype = i32
         lib.lbp_backward_fullrank.argtypes = [vp, vp, vp, vp, vp, C.POINTER(Layer), vp, sz, vp]
         lib.lbp_backward_fullrank.restype = i32
         lib.lbp_poll_status.argtypes = [vp, vp]
@@ -102,7 +106,8 @@ EXPORTED = ("lbp_select_bases", "lbp_basis_matrix", "lbp_flops", "lbp_status_str
             "lbp_last_cuda_error", "lbp_workspace_bytes", "lbp_status_bytes", "lbp_project",
             "lbp_expand", "lbp_backward", "lbp_backward_fullrank", "lbp_poll_status",
             "lbp_backward_static", "lbp_launch_count", "lbp_set_phase_events", "lbp_phase_count",
-            "lbp_phase_name", "lbp_select_lhe", "lbp_spectrum_workspace_bytes", "lbp_spectrum")
+            "lbp_phase_name", "lbp_select_lhe", "lbp_spectrum_workspace_bytes", "lbp_spectrum",
+            "lbp_backward_batch")
 
 
 def _check(status: int, where: str) -> None:
@@ -269,6 +274,27 @@ def lbp_backward(x, g_y, W, k: int, bases, *, gw_dtype: torch.dtype = torch.floa
                                _dev(ws, "ws"), ws.numel(), _stream()),
            "lbp_backward")
     return g_x, g_W
+
+
+def lbp_backward_batch(xs, g_ys, Ws, k: int, bases, *, g_xs, g_Ws, wss):
+    """Algorithm 1 for several independent layers in one call (same k and bases).
+    Every argument is a list with one tensor per layer; outputs and workspaces are
+    the caller's and must not overlap anything of another layer."""
+    n = len(xs)
+    lays = (Layer * n)()
+    for i in range(n):
+        B, H, Wd, Cin = xs[i].shape
+        lays[i] = _layer(B, H, Wd, Cin, g_ys[i].shape[-1], k, _dtype_code(xs[i].dtype),
+                         _dtype_code(g_Ws[i].dtype))
+
+    def ptrs(ts, name):
+        return (C.c_void_p * n)(*[_dev(t, name) for t in ts])
+    sizes = (C.c_size_t * n)(*[w.numel() for w in wss])
+    _check(_lib().lbp_backward_batch(n, ptrs(xs, "x"), ptrs(g_ys, "g_y"), ptrs(Ws, "W"),
+                                     ptrs(g_xs, "g_x"), ptrs(g_Ws, "g_W"), lays, _bases(bases),
+                                     len(bases), ptrs(wss, "ws"), sizes, _stream()),
+           "lbp_backward_batch")
+    return g_xs, g_Ws
 
 
 def lbp_backward_fullrank(x, g_y, W, k: int, *, gw_dtype: torch.dtype = torch.float32,

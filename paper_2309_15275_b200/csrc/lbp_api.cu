@@ -276,20 +276,84 @@ int lbp_expand(const void* t_hat, void* t, int B, int H, int W, int C, int k,
                        RowMap{1, r}, static_cast<cudaStream_t>(stream));
 }
 
-int lbp_backward(const void* x, const void* g_y, const void* W, void* g_x, void* g_W,
-                 const lbp_layer* layer, const lbp_basis* set, int r, void* ws, size_t ws_bytes,
-                 void* stream) {
+// Host-side checks of one lbp_backward problem; nothing is enqueued.
+static int validate_backward(const void* x, const void* g_y, const void* W, const void* g_x,
+                             const void* g_W, const lbp_layer* layer, const lbp_basis* set, int r,
+                             const void* ws, size_t ws_bytes, BasisPlan* plan, Layout* lay) {
   if (x == nullptr || g_y == nullptr || W == nullptr || g_x == nullptr || g_W == nullptr)
     return LBP_ERR_NULL;
   if (int e = check_layer(layer)) return e;
-  const lbp_layer& L = *layer;
-  BasisPlan plan;
-  if (int e = make_basis_plan(L.k, set, r, &plan)) return e;
+  if (int e = make_basis_plan(layer->k, set, r, plan)) return e;
   if (!aligned16(x) || !aligned16(g_y) || !aligned16(W) || !aligned16(g_x) || !aligned16(g_W) ||
       !aligned16(ws))
     return LBP_ERR_ALIGN;
-  const Layout lay = plan_layout(L, r);
-  if (ws == nullptr || ws_bytes < lay.total) return LBP_ERR_WORKSPACE;
+  *lay = plan_layout(*layer, r);
+  if (ws == nullptr || ws_bytes < lay->total) return LBP_ERR_WORKSPACE;
+  return LBP_OK;
+}
+
+int lbp_backward_batch(int n, const void* const* x, const void* const* g_y, const void* const* W,
+                       void* const* g_x, void* const* g_W, const lbp_layer* layers,
+                       const lbp_basis* set, int r, void* const* ws, const size_t* ws_bytes,
+                       void* stream) {
+  if (n < 1 || n > 64) return LBP_ERR_SHAPE;
+  if (x == nullptr || g_y == nullptr || W == nullptr || g_x == nullptr || g_W == nullptr ||
+      layers == nullptr || ws == nullptr || ws_bytes == nullptr)
+    return LBP_ERR_NULL;
+  struct Range {
+    uintptr_t lo, hi;
+  };
+  auto range = [](const void* p, size_t bytes) {
+    const uintptr_t lo = reinterpret_cast<uintptr_t>(p);
+    return Range{lo, lo + bytes};
+  };
+  auto overlap = [](const Range& a, const Range& b) { return a.lo < b.hi && b.lo < a.hi; };
+  Range in[64][3], out[64][3];
+  for (int i = 0; i < n; ++i) {
+    BasisPlan plan;
+    Layout lay;
+    if (int e = validate_backward(x[i], g_y[i], W[i], g_x[i], g_W[i], &layers[i], set, r, ws[i],
+                                  ws_bytes[i], &plan, &lay))
+      return e;
+    const lbp_layer& L = layers[i];
+    const size_t T = static_cast<size_t>(L.B) * L.H * L.W, es = elem_size(L.dtype);
+    in[i][0] = range(x[i], T * L.Cin * es);
+    in[i][1] = range(g_y[i], T * L.Cout * es);
+    in[i][2] = range(W[i], static_cast<size_t>(L.Cout) * L.Cin * es);
+    out[i][0] = range(g_x[i], T * L.Cin * es);
+    out[i][1] = range(g_W[i], static_cast<size_t>(L.Cout) * L.Cin * elem_size(L.gw_dtype));
+    out[i][2] = range(ws[i], lay.total);
+  }
+  // what one problem writes, no other problem may read or write
+  for (int i = 0; i < n; ++i)
+    for (int j = 0; j < n; ++j) {
+      if (i == j) continue;
+      for (int a = 0; a < 3; ++a)
+        for (int b = 0; b < 3; ++b)
+          if (overlap(out[i][a], in[j][b]) || (i < j && overlap(out[i][a], out[j][b])))
+            return LBP_ERR_OVERLAP;
+    }
+  int status = LBP_OK;
+  for (int i = 0; i < n && status == LBP_OK; ++i) {
+    // From the second problem on, the projection kernel need not wait for the
+    // kernel ahead of it (the previous problem's products kernel): it starts on
+    // the SMs that kernel has already left.
+    set_projection_defer_wait(i > 0);
+    status = lbp_backward(x[i], g_y[i], W[i], g_x[i], g_W[i], &layers[i], set, r, ws[i],
+                          ws_bytes[i], stream);
+  }
+  set_projection_defer_wait(false);
+  return status;
+}
+
+int lbp_backward(const void* x, const void* g_y, const void* W, void* g_x, void* g_W,
+                 const lbp_layer* layer, const lbp_basis* set, int r, void* ws, size_t ws_bytes,
+                 void* stream) {
+  BasisPlan plan;
+  Layout lay;
+  if (int e = validate_backward(x, g_y, W, g_x, g_W, layer, set, r, ws, ws_bytes, &plan, &lay))
+    return e;
+  const lbp_layer& L = *layer;
   if (int e = check_device_arch()) return e;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* wsb = static_cast<uint8_t*>(ws);

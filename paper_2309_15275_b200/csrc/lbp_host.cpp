@@ -20,6 +20,10 @@ void note_cuda_failure(cudaError_t e, const char* file, int line) {
     std::fprintf(stderr, "lbp: CUDA error %d at %s:%d\n", static_cast<int>(e), file, line);
 }
 
+thread_local bool g_defer_wait = false;
+void set_projection_defer_wait(bool on) { g_defer_wait = on; }
+bool projection_defer_wait() { return g_defer_wait; }
+
 thread_local long long g_launches = 0;
 void count_launch(int n) { g_launches += n; }
 
@@ -201,6 +205,7 @@ const char* lbp_status_string(int status) {
     case LBP_ERR_CUDA: return "CUDA call failed";
     case LBP_ERR_TIMEOUT: return "bounded device wait expired";
     case LBP_ERR_CAPACITY: return "output array too small";
+    case LBP_ERR_OVERLAP: return "buffers of different problems of a batch overlap";
     default: return "unknown status";
   }
 }

@@ -91,6 +91,10 @@ struct RowMap {
 int launch_project(const void* t, void* t_hat, int dtype, int B, int H, int W, int C,
                    const BasisPlan& plan, RowMap rows, uint32_t* status, cudaStream_t stream);
 
+// Per-thread switch read by the projection launchers (see ProjParams::defer_wait).
+void set_projection_defer_wait(bool on);
+bool projection_defer_wait();
+
 // Projects two tensors that share the token grid (x and g_y) in one launch.
 int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* out1, int C1,
                     int dtype, int B, int H, int W, const BasisPlan& plan, RowMap rows,

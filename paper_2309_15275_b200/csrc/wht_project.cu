@@ -286,6 +286,7 @@ int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* ou
   p.n_items = static_cast<uint32_t>(n0 + n1);
   p.status = status;
   p.scale = 1.0f / static_cast<float>(K);
+  p.defer_wait = projection_defer_wait() ? 1 : 0;
 
   int dev = 0, sms = 0;
   LBP_CUDA_TRY(cudaGetDevice(&dev));

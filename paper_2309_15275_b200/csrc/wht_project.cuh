@@ -18,6 +18,10 @@ struct ProjParams {
   uint32_t n_items0, n_items;   // nb * n_chunks[0], nb * (n_chunks[0] + n_chunks[1])
   uint32_t* status;
   float scale;                  // 1/k
+  // 0: wait for the preceding kernel on the stream before the first access;
+  // 1: the caller vouches that nothing this kernel touches is touched by that
+  // kernel, and the wait moves to the end (it then only keeps completion ordered)
+  int32_t defer_wait;
 };
 
 template <int K, bool BF16>

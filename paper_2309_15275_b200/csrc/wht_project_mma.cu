@@ -60,8 +60,9 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
   // this kernel itself may have been launched the same way behind an earlier
   // kernel on the stream (the products kernel of the previous call, which still
   // reads the buffers written below): nothing is read or written before that
-  // kernel has completed
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // kernel has completed (unless the caller vouches for disjoint buffers, see
+  // ProjParams::defer_wait)
+  if (!p.defer_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   const uint32_t first = blockIdx.x * NW + warp;
   const uint32_t stride = gridDim.x * NW;
@@ -179,6 +180,8 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
       issue(idx + S, s);
     }
   }
+  // deferred: this grid must not complete before the kernel ahead of it has
+  if (p.defer_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // Order 4: a block is only 16 tokens (2 KB per 64 channels), too little per
@@ -219,7 +222,7 @@ __global__ void __launch_bounds__(kStripWarps * 32, 1)
   }
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   __syncthreads();
-  asm volatile("griddepcontrol.wait;" ::: "memory");   // see wht_project_mma_kernel
+  if (!p.defer_wait) asm volatile("griddepcontrol.wait;" ::: "memory");   // see wht_project_mma_kernel
 
   // items count strips here: p.n_items0 / p.n_items = strips * chunks
   const uint32_t first = blockIdx.x * NW + warp;
@@ -325,6 +328,8 @@ __global__ void __launch_bounds__(kStripWarps * 32, 1)
       issue(idx + S, s);
     }
   }
+  // deferred: this grid must not complete before the kernel ahead of it has
+  if (p.defer_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 static int launch_strip4(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloat16* out1,

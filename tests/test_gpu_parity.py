@@ -328,3 +328,40 @@ def test_autograd_linear_backward_is_algorithm_1(dev, dtype):
     assert rel(xd.grad, wx) <= TOL[dtype]
     assert rel(layer.weight.grad, ww) <= TOL[dtype]
     assert layer.weight.grad.dtype == dtype
+
+
+# ------------------------------------------------------ batch of layers ----
+def test_batch_equals_single_calls_and_rejects_overlap(dev):
+    k, r = 8, 8
+    bases = O.select_bases(k, O.RULE_PREFIX, r)
+    shapes = [(768, 2304), (768, 768), (256, 1024), (64, 64)]   # the last one takes the narrow-layer kernel
+    xs, gys, ws_, singles = [], [], [], []
+    for n, (ci, co) in enumerate(shapes):
+        x = synth.make_tensor((4, 16, 16, ci), ("normal", 1.0), "bf16", case_key=960 + n).to(dev)
+        gy = synth.make_tensor((4, 16, 16, co), ("normal", 0.01), "bf16", case_key=970 + n).to(dev)
+        w = synth.make_tensor((co, ci), ("normal", ci ** -0.5), "bf16", case_key=980 + n).to(dev)
+        xs.append(x), gys.append(gy), ws_.append(w)
+        singles.append(lbp.lbp_backward(x, gy, w, k, bases))
+    g_xs = [torch.empty_like(x) for x in xs]
+    g_Ws = [torch.empty((w.shape[0], w.shape[1]), dtype=torch.float32, device=dev) for w in ws_]
+    wss = [lbp.alloc_workspace(x, gy, k, r) for x, gy in zip(xs, gys)]
+    for _ in range(2):
+        lbp.lbp_backward_batch(xs, gys, ws_, k, bases, g_xs=g_xs, g_Ws=g_Ws, wss=wss)
+    for i in range(len(shapes)):
+        ok_status(wss[i])
+        assert torch.equal(g_xs[i], singles[i][0]) and torch.equal(g_Ws[i], singles[i][1])
+    # against the oracle too (the narrow layer)
+    wx, ww = O.backward_lowrank(f64(xs[3]), f64(gys[3]), f64(ws_[3]), k, bases)
+    assert rel(g_xs[3], wx) <= 2e-2 and rel(g_Ws[3], ww) <= 2e-2
+    # an output of one problem that is an input of another is refused before any launch
+    before = g_xs[1].clone()
+    with pytest.raises(lbp.LbpError) as err:
+        lbp.lbp_backward_batch([xs[0], g_xs[0]], [gys[0], gys[1]], [ws_[0], ws_[1]], k, bases,
+                               g_xs=[g_xs[0], g_xs[1]], g_Ws=[g_Ws[0], g_Ws[1]], wss=[wss[0], wss[1]])
+    assert err.value.status == 12
+    with pytest.raises(lbp.LbpError) as err:   # shared workspace
+        lbp.lbp_backward_batch(xs[:2], gys[:2], ws_[:2], k, bases, g_xs=g_xs[:2], g_Ws=g_Ws[:2],
+                               wss=[wss[0], wss[0]])
+    assert err.value.status in (7, 12)
+    torch.cuda.synchronize()
+    assert torch.equal(g_xs[1], before)
