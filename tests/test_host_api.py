@@ -119,3 +119,47 @@ def test_select_lhe_argument_errors():
     assert err.value.status == 3
     assert lbp.lbp_spectrum_workspace_bytes(2, 16, 16, 64, 8, lbp.LBP_BF16) >= 2 * 16 * 16 * 64 * 2
     assert lbp.lbp_spectrum_workspace_bytes(2, 15, 16, 64, 8, lbp.LBP_BF16) == 0
+
+
+def test_batch_arguments_are_checked_on_the_host_before_any_device_call():
+    # fake (never dereferenced) device addresses: every check below happens on the
+    # host, before the library touches the CUDA runtime
+    from paper_2309_15275_b200 import binding as b
+    lib = b._lib()
+    n, k, r = 2, 8, 8
+    bases = lbp.lbp_select_bases(k, lbp.SEL_PREFIX, r)
+    lays = (b.Layer * n)(b._layer(2, 16, 16, 64, 128, k, lbp.LBP_BF16, lbp.LBP_F32),
+                         b._layer(2, 16, 16, 128, 64, k, lbp.LBP_BF16, lbp.LBP_F32))
+    need = [lbp.lbp_workspace_bytes(2, 16, 16, 64, 128, k, lbp.LBP_BF16, lbp.LBP_F32, r),
+            lbp.lbp_workspace_bytes(2, 16, 16, 128, 64, k, lbp.LBP_BF16, lbp.LBP_F32, r)]
+    MB = 1 << 20
+    base = 1 << 32
+
+    def arr(vals):
+        return (ctypes.c_void_p * n)(*vals)
+
+    def call(x, gy, w, gx, gw, ws, sizes=None):
+        sz = (ctypes.c_size_t * n)(*(sizes or need))
+        return lib.lbp_backward_batch(n, arr(x), arr(gy), arr(w), arr(gx), arr(gw), lays,
+                                      b._bases(bases), r, arr(ws), sz, None)
+
+    x = [base, base + 64 * MB]
+    gy = [base + 8 * MB, base + 72 * MB]
+    w = [base + 16 * MB, base + 80 * MB]
+    gx = [base + 24 * MB, base + 88 * MB]
+    gw = [base + 32 * MB, base + 96 * MB]
+    ws = [base + 40 * MB, base + 104 * MB]
+    # g_x of problem 0 is x of problem 1
+    assert call([x[0], gx[0]], gy, w, gx, gw, ws) == 12
+    # the two problems share an output
+    assert call(x, gy, w, gx, [gw[0], gw[0]], ws) == 12
+    # workspace of problem 1 overlaps g_y of problem 0
+    assert call(x, gy, w, gx, gw, [ws[0], gy[0]]) == 12
+    # shared inputs are allowed: the next check that fails is the workspace size
+    assert call([x[0], x[0] + 0], gy, [w[0], w[0]], gx, gw, ws, sizes=[need[0], 16]) in (2, 7)
+    assert call(x, gy, w, gx, gw, ws, sizes=[need[0], need[1] - 1]) == 7
+    assert call(x, gy, w, [gx[0], gx[1] + 2], gw, ws) == 6          # misaligned pointer
+    assert call(x, gy, w, [gx[0], None], gw, ws) == 1               # null pointer
+    assert lib.lbp_backward_batch(0, arr(x), arr(gy), arr(w), arr(gx), arr(gw), lays,
+                                  b._bases(bases), r, arr(ws), (ctypes.c_size_t * n)(*need), None) == 2
+    assert "overlap" in lbp.lbp_status_string(12)
