@@ -67,6 +67,9 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
   const uint32_t first = blockIdx.x * NW + warp;
   const uint32_t stride = gridDim.x * NW;
   const uint32_t n_my = first < p.n_items ? (p.n_items - first + stride - 1) / stride : 0;
+  // x and g_y are read exactly once: they should not push the coefficients just
+  // written (read back from L2 by the products kernel) or W out of L2
+  const uint64_t stream_once = ptx::l2_policy_evict_first();
 
   auto issue = [&](uint32_t idx, int s) {
     uint32_t item = first + idx * stride;
@@ -76,8 +79,8 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
     const uint32_t blk = item / nch, chunk = item - blk * nch;
     const uint32_t bw = blk % p.Wb, t2 = blk / p.Wb, bh = t2 % p.Hb, b = t2 / p.Hb;
     ptx::mbar_expect_tx(&my_bars[s], static_cast<uint32_t>(Cfg::kTileBytes));
-    ptx::tma_load_4d(my_tiles + s * Cfg::kTileBytes, which ? &tmap1 : &tmap0, &my_bars[s],
-                     chunk * 64, bw * K, bh * K, b);
+    ptx::tma_load_4d_hint(my_tiles + s * Cfg::kTileBytes, which ? &tmap1 : &tmap0, &my_bars[s],
+                          chunk * 64, bw * K, bh * K, b, stream_once);
   };
   if (lane == 0) {
     for (uint32_t i = 0; i < S && i < n_my; ++i) issue(i, i);
