@@ -70,6 +70,8 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
   // x and g_y are read exactly once: they should not push the coefficients just
   // written (read back from L2 by the products kernel) or W out of L2
   const uint64_t stream_once = ptx::l2_policy_evict_first();
+  // the coefficients are read back from L2 by the kernel that follows
+  const uint64_t keep = ptx::l2_policy_evict_last();
 
   auto issue = [&](uint32_t idx, int s) {
     uint32_t item = first + idx * stride;
@@ -160,11 +162,11 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
         const int c = cbase + nt * 8;
         if (c < C) {   // C is a multiple of 8: a group of 8 channels is all in or all out
           if (q0 < p.r)
-            *reinterpret_cast<uint32_t*>(out + (row0 + q0) * C + c) =
-                pack_bf16x2(d[mt][nt][0] * p.scale, d[mt][nt][1] * p.scale);
+            ptx::st_global_hint_u32(out + (row0 + q0) * C + c,
+                                    pack_bf16x2(d[mt][nt][0] * p.scale, d[mt][nt][1] * p.scale), keep);
           if (q1 < p.r)
-            *reinterpret_cast<uint32_t*>(out + (row0 + q1) * C + c) =
-                pack_bf16x2(d[mt][nt][2] * p.scale, d[mt][nt][3] * p.scale);
+            ptx::st_global_hint_u32(out + (row0 + q1) * C + c,
+                                    pack_bf16x2(d[mt][nt][2] * p.scale, d[mt][nt][3] * p.scale), keep);
         }
       }
     }
