@@ -74,12 +74,14 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // TMA load whose completion is signalled on a barrier that may live in the peer CTA
+// `policy`: L2 eviction hint (the operands are read by several pairs, from L2)
 __device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* m,
-                                                 uint32_t bar_cluster_addr, int32_t x, int32_t y) {
+                                                 uint32_t bar_cluster_addr, int32_t x, int32_t y,
+                                                 uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
-      "[%0], [%1, {%3, %4}], [%2];" ::"r"(ptx::smem_u32(smem_dst)),
-      "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster_addr), "r"(x), "r"(y)
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+      ".L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(ptx::smem_u32(smem_dst)),
+      "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster_addr), "r"(x), "r"(y), "l"(policy)
       : "memory");
 }
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_dst, uint32_t ncols) {
@@ -242,6 +244,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       // launched with programmatic stream serialization: x_hat / g_y_hat of the
       // projection kernel may only be read after this wait
       asm volatile("griddepcontrol.wait;" ::: "memory");
+      const uint64_t keep = ptx::l2_policy_evict_last();
       uint32_t it = 0;
       bool ok = true;
       for (int ti = 0; ti < my_tiles && ok; ++ti) {
@@ -261,17 +264,17 @@ __global__ void __launch_bounds__(kThreads, 1)
           const uint32_t bar = map_to_rank(ptx::smem_u32(&full_bar[s]), 0);
           if (tl.is_gw) {
             const int m0 = tl.a * 256 + static_cast<int>(rank) * 128;
-            tma_load_2d_pair(sa, &tm_gyhat_mn, bar, m0, kb * BK);
-            tma_load_2d_pair(sa + kChunkBytes, &tm_gyhat_mn, bar, m0 + 64, kb * BK);
+            tma_load_2d_pair(sa, &tm_gyhat_mn, bar, m0, kb * BK, keep);
+            tma_load_2d_pair(sa + kChunkBytes, &tm_gyhat_mn, bar, m0 + 64, kb * BK, keep);
             const int n0 = tl.b * bn + static_cast<int>(rank) * half;
             for (int c = 0; c < half / 64; ++c)
-              tma_load_2d_pair(sb + c * kChunkBytes, &tm_xhat, bar, n0 + c * 64, kb * BK);
+              tma_load_2d_pair(sb + c * kChunkBytes, &tm_xhat, bar, n0 + c * 64, kb * BK, keep);
           } else {
             const int g = 2 * tl.a + static_cast<int>(rank);
-            tma_load_2d_pair(sa, &tm_gyhat_k, bar, kb * BK, g * BM);
+            tma_load_2d_pair(sa, &tm_gyhat_k, bar, kb * BK, g * BM, keep);
             const int n0 = tl.b * bn + static_cast<int>(rank) * half;
             for (int c = 0; c < half / 64; ++c)
-              tma_load_2d_pair(sb + c * kChunkBytes, &tm_w, bar, n0 + c * 64, kb * BK);
+              tma_load_2d_pair(sb + c * kChunkBytes, &tm_w, bar, n0 + c * 64, kb * BK, keep);
           }
           ++it;
         }
