@@ -179,6 +179,8 @@ __global__ void __launch_bounds__(kThreads, 1)
       // above overlaps the tail of the projection kernel; its results (x_hat,
       // g_y_hat) may only be read after this wait.
       asm volatile("griddepcontrol.wait;" ::: "memory");
+      // the operands are read by several CTAs, from L2
+      const uint64_t keep = ptx::l2_policy_evict_last();
       uint32_t it = 0;
       bool ok = true;
       for (int ti = 0; ti < my_tiles && ok; ++ti) {
@@ -196,16 +198,16 @@ __global__ void __launch_bounds__(kThreads, 1)
           ptx::mbar_expect_tx(&full_bar[s], tx);
           if (tl.is_gw) {
             // A = g_y_hat^T tile: stored (rows, Cout), MN-major, two 64-wide chunks
-            ptx::tma_load_2d(sa, &tm_gyhat_mn, &full_bar[s], tl.a * 128, kb * BK);
-            ptx::tma_load_2d(sa + kChunkBytes, &tm_gyhat_mn, &full_bar[s], tl.a * 128 + 64, kb * BK);
+            ptx::tma_load_2d_hint(sa, &tm_gyhat_mn, &full_bar[s], tl.a * 128, kb * BK, keep);
+            ptx::tma_load_2d_hint(sa + kChunkBytes, &tm_gyhat_mn, &full_bar[s], tl.a * 128 + 64, kb * BK, keep);
             for (int c = 0; c < bn / 64; ++c)
-              ptx::tma_load_2d(sb + c * kChunkBytes, &tm_xhat, &full_bar[s], tl.b * bn + c * 64,
-                               kb * BK);
+              ptx::tma_load_2d_hint(sb + c * kChunkBytes, &tm_xhat, &full_bar[s], tl.b * bn + c * 64,
+                               kb * BK, keep);
           } else {
             // A = g_y_hat rows of group m, K-major
-            ptx::tma_load_2d(sa, &tm_gyhat_k, &full_bar[s], kb * BK, tl.a * BM);
+            ptx::tma_load_2d_hint(sa, &tm_gyhat_k, &full_bar[s], kb * BK, tl.a * BM, keep);
             for (int c = 0; c < bn / 64; ++c)
-              ptx::tma_load_2d(sb + c * kChunkBytes, &tm_w, &full_bar[s], tl.b * bn + c * 64, kb * BK);
+              ptx::tma_load_2d_hint(sb + c * kChunkBytes, &tm_w, &full_bar[s], tl.b * bn + c * 64, kb * BK, keep);
           }
           ++it;
         }

@@ -234,6 +234,8 @@ __global__ void __launch_bounds__(kStripWarps * 32, 1)
   const uint32_t stride = gridDim.x * NW;
   const uint32_t n_my = first < p.n_items ? (p.n_items - first + stride - 1) / stride : 0;
   const uint32_t Wb4 = (static_cast<uint32_t>(p.Wb) + kStripBlocks - 1) / kStripBlocks;
+  const uint64_t stream_once = ptx::l2_policy_evict_first();   // as in wht_project_mma_kernel
+  const uint64_t keep = ptx::l2_policy_evict_last();
 
   auto issue = [&](uint32_t idx, int s) {
     uint32_t item = first + idx * stride;
@@ -244,8 +246,8 @@ __global__ void __launch_bounds__(kStripWarps * 32, 1)
     const uint32_t bw4 = sg % Wb4, t2 = sg / Wb4, bh = t2 % p.Hb, b = t2 / p.Hb;
     ptx::mbar_expect_tx(&my_bars[s], static_cast<uint32_t>(kStripTileBytes));
     // tokens past W (a last strip of fewer than four blocks) are zero-filled
-    ptx::tma_load_4d(my_tiles + s * kStripTileBytes, which ? &tmap1 : &tmap0, &my_bars[s],
-                     chunk * 64, bw4 * (K * kStripBlocks), bh * K, b);
+    ptx::tma_load_4d_hint(my_tiles + s * kStripTileBytes, which ? &tmap1 : &tmap0, &my_bars[s],
+                          chunk * 64, bw4 * (K * kStripBlocks), bh * K, b, stream_once);
   };
   if (lane == 0) {
     for (uint32_t i = 0; i < S && i < n_my; ++i) issue(i, i);
@@ -309,11 +311,11 @@ __global__ void __launch_bounds__(kStripWarps * 32, 1)
           const int c = cbase + nt * 8;
           if (c < C) {
             if (q0 < p.r)
-              *reinterpret_cast<uint32_t*>(out + (row0 + q0) * C + c) =
-                  pack_bf16x2(d[nt][0] * p.scale, d[nt][1] * p.scale);
+              ptx::st_global_hint_u32(out + (row0 + q0) * C + c,
+                                      pack_bf16x2(d[nt][0] * p.scale, d[nt][1] * p.scale), keep);
             if (q1 < p.r)
-              *reinterpret_cast<uint32_t*>(out + (row0 + q1) * C + c) =
-                  pack_bf16x2(d[nt][2] * p.scale, d[nt][3] * p.scale);
+              ptx::st_global_hint_u32(out + (row0 + q1) * C + c,
+                                      pack_bf16x2(d[nt][2] * p.scale, d[nt][3] * p.scale), keep);
           }
         }
         // rows of a padded row tile that no block owns are kept at zero
