@@ -49,7 +49,7 @@ def _peaks():
 # DRAM traffic per step (sum over the four layers, bytes) of the two kernels, from
 # the ncu capture summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum);
 # None = not captured for the current kernels.
-NCU_TRAFFIC_PER_STEP = {"wht_project_mma_kernel": 869.3e6, "lbp_products_pair_kernel": 282.9e6}
+NCU_TRAFFIC_PER_STEP = {"wht_project_mma_kernel": 830.1e6, "lbp_products_pair_kernel": 285.2e6}
 
 
 # ------------------------------------------------------------------ clocks ----
