@@ -328,8 +328,10 @@ def run_gpu(args):
             wss = [lbp.alloc_workspace(L["x"], L["gy"], k, rr) for L in layers]
 
             def one_step():
-                for L, w_ in zip(layers, wss):
-                    lbp.lbp_backward(L["x"], L["gy"], L["w"], k, bases_r, g_x=L["gx"], g_W=L["gw"], ws=w_)
+                lbp.lbp_backward_batch([L["x"] for L in layers], [L["gy"] for L in layers],
+                                       [L["w"] for L in layers], k, bases_r,
+                                       g_xs=[L["gx"] for L in layers], g_Ws=[L["gw"] for L in layers],
+                                       wss=wss)
             for _ in range(3):
                 one_step()
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
