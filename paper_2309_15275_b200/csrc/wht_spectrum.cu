@@ -60,13 +60,15 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
   const uint32_t stride = gridDim.x * NW;
   const uint32_t n_my = first < p.n_items ? (p.n_items - first + stride - 1) / stride : 0;
   const uint32_t nch = static_cast<uint32_t>(p.n_chunks[0]);
+  const uint64_t stream_once = ptx::l2_policy_evict_first();   // the tensor is read exactly once
 
   auto issue = [&](uint32_t idx, int s) {
     const uint32_t item = first + idx * stride;
     const uint32_t blk = item / nch, chunk = item - blk * nch;
     const uint32_t bw = blk % p.Wb, t2 = blk / p.Wb, bh = t2 % p.Hb, b = t2 / p.Hb;
     ptx::mbar_expect_tx(&my_bars[s], static_cast<uint32_t>(Cfg::kTileBytes));
-    ptx::tma_load_4d(my_tiles + s * Cfg::kTileBytes, &tmap, &my_bars[s], chunk * 64, bw * K, bh * K, b);
+    ptx::tma_load_4d_hint(my_tiles + s * Cfg::kTileBytes, &tmap, &my_bars[s], chunk * 64, bw * K, bh * K, b,
+                          stream_once);
   };
   if (lane == 0) {
     for (uint32_t i = 0; i < S && i < n_my; ++i) issue(i, i);
