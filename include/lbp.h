@@ -137,7 +137,7 @@ int lbp_project(const void* t, void* t_hat, int B, int H, int W, int C, int k,
  *   energy[i*k + j] = sum over blocks and channels of t_hat[.., (i,j), ..]^2
  * with t_hat the coefficients of Eq. 6 for all k*k bases, so that the k*k
  * energies add up to ||t||^2.  t (B,H,W,C) of `dtype`; energy: DEVICE array of
- * k*k doubles, overwritten.  bf16 data of order 4 or 8: one pass over t, fp32
+ * k*k doubles, overwritten.  bf16 data: one pass over t, fp32
  * responses squared and summed in fp32 per thread, fp64 across threads, and
  * the workspace holds only the status block.  Otherwise the coefficients are
  * materialised in `dtype` (fp32 accumulation, one rounding) in the workspace

@@ -167,7 +167,142 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
   for (int i = threadIdx.x; i < R; i += NW * 32) atomicAdd(&energy[i], e_sm[i] * s2);
 }
 
-bool spectrum_mma_supported(int k, int dtype) { return dtype == LBP_BF16 && (k == 4 || k == 8); }
+// ---- one pass: bf16 data, k = 16 --------------------------------------------
+// 256 responses per block are too many rows for the dense form above (4x the
+// MMA work per byte of order 8).  The 2-D transform is separable: the transform
+// along W (v) is a 16 x 16 Hadamard matrix applied by warp MMA to each of the 16
+// token rows u of the block, one 8-channel n-tile at a time; the transform along H
+// (u) is then a 16-point butterfly across the 16 accumulator sets, which a thread
+// holds for the same (row, channel) positions.  Both in natural (Sylvester) order;
+// `seq_of_nat` turns natural indices into sequency indices for the result.
+struct Seq16 {
+  uint8_t seq_of_nat[16];
+};
+
+__device__ __forceinline__ void ldmatrix_x2_trans(uint32_t addr, uint32_t& r0, uint32_t& r1) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];"
+               : "=r"(r0), "=r"(r1)
+               : "r"(addr)
+               : "memory");
+}
+
+__global__ void __launch_bounds__(MmaCfg<16>::kWarps * 32, 1)
+    wht_spectrum16_kernel(const __grid_constant__ CUtensorMap tmap,
+                          const __grid_constant__ ProjParams p, const __grid_constant__ Seq16 sq,
+                          double* __restrict__ energy) {
+  using Cfg = MmaCfg<16>;
+  constexpr int K = 16, NW = Cfg::kWarps, S = Cfg::kStages, R = K * K;
+
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ double e_sm[R];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + NW * S * Cfg::kTileBytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, tq = lane & 3;
+  uint64_t* my_bars = bars + warp * S;
+  uint8_t* my_tiles = tiles + warp * S * Cfg::kTileBytes;
+
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < S; ++s) ptx::mbar_init(&my_bars[s], 1);
+    ptx::mbar_fence_init();
+  }
+  if (threadIdx.x == 0) ptx::prefetch_tensormap(&tmap);
+  for (int i = threadIdx.x; i < R; i += NW * 32) e_sm[i] = 0.0;
+  __syncthreads();
+
+  const uint32_t first = blockIdx.x * NW + warp;
+  const uint32_t stride = gridDim.x * NW;
+  const uint32_t n_my = first < p.n_items ? (p.n_items - first + stride - 1) / stride : 0;
+  const uint32_t nch = static_cast<uint32_t>(p.n_chunks[0]);
+  const uint64_t stream_once = ptx::l2_policy_evict_first();
+
+  auto issue = [&](uint32_t idx, int s) {
+    const uint32_t item = first + idx * stride;
+    const uint32_t blk = item / nch, chunk = item - blk * nch;
+    const uint32_t bw = blk % p.Wb, t2 = blk / p.Wb, bh = t2 % p.Hb, b = t2 / p.Hb;
+    ptx::mbar_expect_tx(&my_bars[s], static_cast<uint32_t>(Cfg::kTileBytes));
+    ptx::tma_load_4d_hint(my_tiles + s * Cfg::kTileBytes, &tmap, &my_bars[s], chunk * 64, bw * K, bh * K, b,
+                          stream_once);
+  };
+  if (lane == 0) {
+    for (uint32_t i = 0; i < S && i < n_my; ++i) issue(i, i);
+  }
+
+  // A = natural-order Hadamard matrix H[b][v] = (-1)^popcount(b & v), m16 x k16
+  uint32_t afrag[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int b = g + (j & 1) * 8;
+    const int v = 2 * tq + (j >> 1) * 8;
+    const uint32_t lo = (__popc(b & v) & 1) ? 0xBF80u : 0x3F80u;
+    const uint32_t hi = (__popc(b & (v + 1)) & 1) ? 0xBF80u : 0x3F80u;
+    afrag[j] = lo | (hi << 16);
+  }
+
+  // e[a][h]: natural row index a of the transform along H, column index g + 8 h
+  float e[K][2];
+#pragma unroll
+  for (int a = 0; a < K; ++a) e[a][0] = e[a][1] = 0.f;
+
+  // ldmatrix.x2.trans: lanes 0-15 give the rows; matrices 0 / 1 are v = 0..7 / 8..15
+  const int ld_v = ((lane >> 3) & 1) * 8 + (lane & 7);
+
+  for (uint32_t idx = 0; idx < n_my; ++idx) {
+    const int s = static_cast<int>(idx % S);
+    const uint32_t parity = (idx / S) & 1u;
+    const bool ok = ptx::mbar_wait(&my_bars[s], parity, p.status, (6u << 16) | 2u);
+    if (!__all_sync(0xffffffffu, ok)) break;
+    const uint32_t tile = ptx::smem_u32(my_tiles + s * Cfg::kTileBytes);
+
+#pragma unroll 1
+    for (int nt = 0; nt < 8; ++nt) {
+      float dd[4][K];   // [fragment position][u]
+#pragma unroll
+      for (int u = 0; u < K; ++u) {
+        const int row = u * K + ld_v;
+        uint32_t b0, b1;
+        ldmatrix_x2_trans(tile + row * 128 + ((nt ^ (row & 7)) << 4), b0, b1);
+        float d[4] = {0.f, 0.f, 0.f, 0.f};
+        mma_bf16_16816(d, afrag, b0, b1);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) dd[j][u] = d[j];
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        hadamard_vec<K>(dd[j]);
+#pragma unroll
+        for (int a = 0; a < K; ++a) e[a][j >> 1] = fmaf(dd[j][a], dd[j][a], e[a][j >> 1]);
+      }
+    }
+
+    __syncwarp();
+    if (lane == 0 && idx + S < n_my) {
+      ptx::fence_proxy_async_smem();
+      issue(idx + S, s);
+    }
+  }
+
+#pragma unroll
+  for (int a = 0; a < K; ++a)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      float v = e[a][h];
+      v += __shfl_xor_sync(0xffffffffu, v, 1);
+      v += __shfl_xor_sync(0xffffffffu, v, 2);
+      if (tq == 0)
+        atomicAdd(&e_sm[sq.seq_of_nat[a] * K + sq.seq_of_nat[g + 8 * h]], static_cast<double>(v));
+    }
+  __syncthreads();
+  const double s2 = static_cast<double>(p.scale) * static_cast<double>(p.scale);
+  for (int i = threadIdx.x; i < R; i += NW * 32) atomicAdd(&energy[i], e_sm[i] * s2);
+}
+
+bool spectrum_mma_supported(int k, int dtype) {
+  return dtype == LBP_BF16 && (k == 4 || k == 8 || k == 16);
+}
 
 template <int K>
 static int launch_spectrum_mma_k(const CUtensorMap& tmap, const ProjParams& p, const MmaPlan& mp,
@@ -212,6 +347,19 @@ int launch_spectrum_mma(const void* t, int B, int H, int W, int C, const BasisPl
   int dev = 0, sms = 0;
   LBP_CUDA_TRY(cudaGetDevice(&dev));
   LBP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  if (K == 16) {
+    Seq16 sq;
+    for (int sidx = 0; sidx < 16; ++sidx) sq.seq_of_nat[walsh_natural_index(16, sidx)] = static_cast<uint8_t>(sidx);
+    using Cfg = MmaCfg<16>;
+    LBP_CUDA_TRY(cudaFuncSetAttribute(wht_spectrum16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      Cfg::kSmemBytes));
+    const uint32_t want = (p.n_items + Cfg::kWarps - 1) / Cfg::kWarps;
+    const int grid = static_cast<int>(want < static_cast<uint32_t>(sms) ? want : sms);
+    wht_spectrum16_kernel<<<grid, Cfg::kWarps * 32, Cfg::kSmemBytes, stream>>>(tmap, p, sq, energy);
+    count_launch();
+    LBP_CUDA_TRY(cudaGetLastError());
+    return LBP_OK;
+  }
   if (K == 4) return launch_spectrum_mma_k<4>(tmap, p, mp, energy, sms, stream);
   return launch_spectrum_mma_k<8>(tmap, p, mp, energy, sms, stream);
 }
