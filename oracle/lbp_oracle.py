@@ -28,6 +28,8 @@ Parity status: every function below is pinned by tests/test_oracle_pins.py
 special cases, the paper's printed ranks and FLOP figures), except
 `lowrank error vs exact BP at r < k^2`, for which the paper gives no bound:
 "parity unpinned" for that quantity only (it is not an output of the path).
+The variants for real ViT token maps (zero-extended grids, tokens outside the
+grid, bias gradient, accumulation, x_hat handed in) are pinned there too.
 """
 from __future__ import annotations
 
@@ -239,6 +241,89 @@ def backward_lowrank(x, g_y, w, k: int, bases):
 
 
 # --------------------------------------------------------------------------
+# Variants of Algorithm 1 that a ViT needs around its token grid.  The paper
+# does not describe them; each docstring states the reading taken.
+# --------------------------------------------------------------------------
+def backward_lowrank_projected(x_hat, g_y, w, k: int, bases):
+    """Algorithm 1 from its second step on, with x_hat = p(x) (Eq. 3) handed in
+    instead of x: the projection of x can be taken at forward time and only its
+    r/k^2 coefficients kept.
+
+    x_hat (B, H/k, W/k, r, Cx) in the order of `bases`; g_y (B, H, W, Cy).
+    g_y_hat <- p(g_y); g_w <- g_y_hat^T x_hat; g_x_hat <- g_y_hat w;
+    g_x <- p^{-1}(g_x_hat).
+    """
+    _check_bases(k, bases)
+    x_hat = np.asarray(x_hat, dtype=np.float64)
+    w = np.asarray(w, dtype=np.float64)
+    gy_hat = project(g_y, k, bases)
+    if x_hat.shape[:4] != gy_hat.shape[:4]:
+        raise ValueError("x_hat does not match the block grid of g_y")
+    Cin, Cout = x_hat.shape[-1], gy_hat.shape[-1]
+    g_w = gy_hat.reshape(-1, Cout).T @ x_hat.reshape(-1, Cin)
+    g_x = expand(gy_hat @ w, k, bases)
+    return g_x, g_w
+
+
+def pad_grid(t, k: int) -> np.ndarray:
+    """Reading for token grids whose sides are not multiples of the order k (the
+    paper's 7 x 7 maps, L = 49, under an order-8 transform): the grid is
+    extended with zero tokens at its high end (bottom rows, right columns) to
+    the next multiple of k; blocks stay aligned at the origin."""
+    t = np.asarray(t, dtype=np.float64)
+    B, H, W, C = t.shape
+    Hp, Wp = -(-H // k) * k, -(-W // k) * k
+    out = np.zeros((B, Hp, Wp, C), dtype=np.float64)
+    out[:, :H, :W, :] = t
+    return out
+
+
+def project_padded(t, k: int, bases) -> np.ndarray:
+    """Eq. 6 on the zero-extended grid: (B,H,W,C) -> (B, ceil(H/k), ceil(W/k), r, C)."""
+    return project(pad_grid(t, k), k, bases)
+
+
+def backward_lowrank_padded(x, g_y, w, k: int, bases):
+    """Algorithm 1 on the zero-extended grid; g_x is returned for the real tokens
+    only (the gradient of a padding token has no consumer).  The zero tokens add
+    nothing to g_w."""
+    x = np.asarray(x, dtype=np.float64)
+    B, H, W, _ = x.shape
+    g_x, g_w = backward_lowrank(pad_grid(x, k), pad_grid(g_y, k), w, k, bases)
+    return g_x[:, :H, :W, :], g_w
+
+
+def backward_extra_tokens(x_extra, gy_extra, w):
+    """Tokens that are not part of the grid (a class token): the paper's method
+    has nothing to say about them, so they take vanilla BP (Eq. 2) exactly.
+    x_extra (n, Cx), gy_extra (n, Cy) -> (g_x_extra (n, Cx), their term of g_w)."""
+    x_extra = np.asarray(x_extra, dtype=np.float64)
+    gy_extra = np.asarray(gy_extra, dtype=np.float64)
+    w = np.asarray(w, dtype=np.float64)
+    return gy_extra @ w, gy_extra.T @ x_extra
+
+
+def bias_grad(g_y, gy_extra=None) -> np.ndarray:
+    """Gradient of a bias added to y (Eq. 1 has none; every ViT linear has one):
+    the sum of g_y over all tokens, exact.  For the grid tokens this equals
+    k * sum over blocks of the (0,0) coefficient of g_y_hat."""
+    g_y = np.asarray(g_y, dtype=np.float64)
+    out = g_y.reshape(-1, g_y.shape[-1]).sum(axis=0)
+    if gy_extra is not None:
+        gy_extra = np.asarray(gy_extra, dtype=np.float64)
+        out = out + gy_extra.reshape(-1, gy_extra.shape[-1]).sum(axis=0)
+    return out
+
+
+def accumulate(g_w_new, g_w_prev=None, beta: float = 0.0) -> np.ndarray:
+    """g_w <- beta * g_w_prev + g_w_new (gradient accumulation over micro-batches)."""
+    g_w_new = np.asarray(g_w_new, dtype=np.float64)
+    if g_w_prev is None or beta == 0.0:
+        return g_w_new
+    return beta * np.asarray(g_w_prev, dtype=np.float64) + g_w_new
+
+
+# --------------------------------------------------------------------------
 # Cost model (Table 1)
 # --------------------------------------------------------------------------
 def flops(Cx: int, Cy: int, L: int, r: int) -> dict:
@@ -258,3 +343,30 @@ def rel_fro(a, b) -> float:
     den = np.linalg.norm(b.ravel())
     num = np.linalg.norm((a - b).ravel())
     return float(num / den) if den > 0 else float(num)
+
+
+def block_rel_fro(a, b, k: int) -> float:
+    """Largest relative Frobenius error over the k x k token blocks of a
+    (B,H,W,C) tensor (H, W multiples of k): a wrong patch cannot hide in the
+    norm of the whole tensor.  Blocks whose reference is all zero count with
+    their absolute error."""
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    d = to_blocks(a - b, k)
+    num = np.sqrt(np.sum(d * d, axis=(3, 4)))
+    rb = to_blocks(b, k)
+    den = np.sqrt(np.sum(rb * rb, axis=(3, 4)))
+    ratio = np.where(den > 0, num / np.where(den > 0, den, 1.0), num)
+    return float(ratio.max())
+
+
+def tile_rel_fro(a, b, tile: int = 128) -> float:
+    """Largest relative Frobenius error over tile x tile pieces of a matrix
+    (ragged edge pieces included)."""
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    worst = 0.0
+    for i in range(0, b.shape[0], tile):
+        for j in range(0, b.shape[1], tile):
+            worst = max(worst, rel_fro(a[i:i + tile, j:j + tile], b[i:i + tile, j:j + tile]))
+    return worst

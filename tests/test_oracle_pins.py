@@ -492,3 +492,186 @@ def test_lhe_on_a_decaying_spectrum_equals_the_low_pass_set():
     for r in (1, 3, 8, 10, 21):
         assert O.select_lhe(E, k, r) == order[:r]
     assert set(O.select_lhe(E, k, 10)) == set(O.select_bases(k, O.RULE_L1, 4))
+
+
+# ------------------------------------------------------- error measures ----
+def test_rel_fro_is_the_relative_frobenius_error():
+    # every parity assertion goes through these: pin them to hand-computed values
+    b = np.array([[3.0, 4.0], [0.0, 12.0]])                      # ||b|| = 13
+    assert O.rel_fro(b * (1 + 1e-3), b) == pytest.approx(1e-3, rel=1e-12)
+    assert O.rel_fro(b + np.array([[0.0, 0.0], [5.0, 0.0]]), b) == pytest.approx(5.0 / 13.0, rel=1e-12)
+    assert O.rel_fro(np.array([1.0, 0.0]), np.array([0.0, 1.0])) == pytest.approx(np.sqrt(2.0))
+    assert O.rel_fro(b, b) == 0.0
+    # the reference is the second argument (the denominator)
+    assert O.rel_fro(2 * b, b) == pytest.approx(1.0) and O.rel_fro(b, 2 * b) == pytest.approx(0.5)
+    # zero reference: the absolute error
+    assert O.rel_fro(np.array([3.0, 4.0]), np.zeros(2)) == pytest.approx(5.0)
+
+
+def test_local_error_measures_find_one_bad_patch():
+    k = 4
+    rng = np.random.default_rng(21)
+    ref = rng.standard_normal((2, 2 * k, 3 * k, 5))
+    got = ref.copy()
+    got[1, k:2 * k, 2 * k:3 * k, :] *= 1.5                        # one block off by 50 %
+    assert O.block_rel_fro(got, ref, k) == pytest.approx(0.5, rel=1e-12)
+    assert O.rel_fro(got, ref) < 0.25                             # diluted in the global norm
+    assert O.block_rel_fro(ref, ref, k) == 0.0
+    m = rng.standard_normal((300, 200))
+    bad = m.copy()
+    bad[256:300, 128:200] *= 3.0                                  # the ragged corner tile
+    assert O.tile_rel_fro(bad, m, 128) == pytest.approx(2.0, rel=1e-12)
+    assert O.rel_fro(bad, m) < 1.0
+    bad2 = m.copy()
+    bad2[0, 0] += 1.0
+    t00 = np.linalg.norm(m[:128, :128])
+    assert O.tile_rel_fro(bad2, m, 128) == pytest.approx(1.0 / t00, rel=1e-12)
+
+
+# ------------------------------------- x_hat handed in (Eq. 3, Alg. 1) ----
+@pytest.mark.parametrize("k,r", [(4, 5), (8, 8), (16, 3)])
+def test_projected_backward_is_vanilla_bp_on_the_expanded_coefficients(k, r):
+    # g_w = g_y_hat^T x_hat = (P^T g_y)^T x_hat = g_y^T (P x_hat): Eq. 2 with x
+    # replaced by p^{-1}(x_hat), for ANY coefficient tensor (not only projections)
+    rng = np.random.default_rng(31 + k)
+    bases = O.select_bases(k, O.RULE_PREFIX, r)
+    B, Hb, Wb, Cin, Cout = 2, 2, 1, 5, 4
+    x_hat = rng.standard_normal((B, Hb, Wb, r, Cin))
+    gy = rng.standard_normal((B, Hb * k, Wb * k, Cout))
+    w = rng.standard_normal((Cout, Cin))
+    gx, gw = O.backward_lowrank_projected(x_hat, gy, w, k, bases)
+    _, gw_ref = O.backward_exact(O.expand(x_hat, k, bases), gy, w)
+    assert np.allclose(gw, gw_ref, rtol=1e-12, atol=1e-12)
+    # g_x does not depend on x_hat: the dense projector applied to g_y w
+    P = O.basis_matrix(k, bases).astype(np.float64) / k
+    Pi = P @ P.T
+    exact_gx = O.to_blocks((gy.reshape(-1, Cout) @ w).reshape(B, Hb * k, Wb * k, Cin), k)
+    want = O.from_blocks(np.einsum("pq,bhwqc->bhwpc", Pi, exact_gx), k)
+    assert np.allclose(gx, want, rtol=1e-12, atol=1e-12)
+
+
+def test_projected_backward_equals_algorithm_1_when_x_hat_is_p_of_x():
+    k, r = 8, 10
+    x, gy, w = _tiny(k, 41)
+    bases = O.select_bases(k, O.RULE_PREFIX, r)
+    a = O.backward_lowrank(x, gy, w, k, bases)
+    b = O.backward_lowrank_projected(O.project(x, k, bases), gy, w, k, bases)
+    assert np.allclose(a[0], b[0], atol=1e-13) and np.allclose(a[1], b[1], atol=1e-12)
+    with pytest.raises(ValueError):
+        O.backward_lowrank_projected(O.project(x, k, bases)[:, :1], gy, w, k, bases)
+
+
+# ------------------------------------ grids that are not multiples of k ----
+def test_padding_goes_to_the_high_end_of_the_grid():
+    # a single token at the last real position (6, 6) of a 7 x 7 map, order 8:
+    # its coefficients are wal_i[6] wal_j[6] / 8 -- it sits at (6, 6) of the block,
+    # so the zero tokens were appended after it, not before
+    k = 8
+    t = np.zeros((1, 7, 7, 1))
+    t[0, 6, 6, 0] = 2.0
+    pairs = [(i, j) for i in range(k) for j in range(k)]
+    th = O.project_padded(t, k, pairs)
+    assert th.shape == (1, 1, 1, 64, 1)
+    wal = O.walsh(k)
+    want = np.array([wal[i][6] * wal[j][6] * 2.0 / k for (i, j) in pairs])
+    assert np.allclose(th[0, 0, 0, :, 0], want, atol=1e-15)
+    assert O.pad_grid(t, k).shape == (1, 8, 8, 1) and O.pad_grid(t, k)[0, 7, 7, 0] == 0.0
+    assert O.pad_grid(np.ones((1, 8, 16, 2)), 8).shape == (1, 8, 16, 2)
+
+
+@pytest.mark.parametrize("k,H,W", [(8, 7, 7), (4, 7, 7), (8, 14, 14), (4, 6, 9)])
+def test_padded_full_rank_is_exact_bp_on_the_real_tokens(k, H, W):
+    rng = np.random.default_rng(50 + k + H)
+    x = rng.standard_normal((2, H, W, 6))
+    gy = rng.standard_normal((2, H, W, 3))
+    w = rng.standard_normal((3, 6))
+    pairs = O.select_bases(k, O.RULE_PREFIX, k * k)
+    gx, gw = O.backward_lowrank_padded(x, gy, w, k, pairs)
+    ex, ew = O.backward_exact(x, gy, w)
+    assert gx.shape == x.shape
+    assert np.allclose(gx, ex, atol=1e-12) and np.allclose(gw, ew, atol=1e-11)
+
+
+def test_padded_rank1_pools_over_the_real_tokens_of_a_block():
+    # r = 1 (DC only): every real token of a block receives
+    # (sum of g_y over the block's real tokens / k^2) w, partial blocks included
+    k, H, W = 4, 6, 7
+    rng = np.random.default_rng(61)
+    x = rng.standard_normal((1, H, W, 3))
+    gy = rng.standard_normal((1, H, W, 2))
+    w = rng.standard_normal((2, 3))
+    gx, gw = O.backward_lowrank_padded(x, gy, w, k, [(0, 0)])
+    want_w = np.zeros((2, 3))
+    for bh in range(2):
+        for bw in range(2):
+            hs, ws_ = slice(bh * k, min(H, bh * k + k)), slice(bw * k, min(W, bw * k + k))
+            sg = gy[0, hs, ws_].reshape(-1, 2).sum(axis=0)
+            sx = x[0, hs, ws_].reshape(-1, 3).sum(axis=0)
+            assert np.allclose(gx[0, hs, ws_], (sg / (k * k)) @ w, atol=1e-13)
+            want_w += np.outer(sg, sx) / (k * k)
+    assert np.allclose(gw, want_w, atol=1e-12)
+
+
+def test_padded_equals_plain_on_divisible_grids():
+    k = 8
+    x, gy, w = _tiny(k, 71)
+    bases = O.select_bases(k, O.RULE_L1, 3)
+    a = O.backward_lowrank(x, gy, w, k, bases)
+    b = O.backward_lowrank_padded(x, gy, w, k, bases)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+
+
+# ------------------------- tokens outside the grid, bias, accumulation ----
+def test_class_token_rows_take_vanilla_bp_and_complete_the_layer():
+    # a (B, 1 + H W, C) ViT tensor: grid tokens at full rank plus the class token
+    # by Eq. 2 must add up to vanilla BP over all 1 + H W tokens
+    k, B, Cin, Cout = 4, 3, 5, 4
+    rng = np.random.default_rng(81)
+    xt = rng.standard_normal((B, 1 + k * k, Cin))
+    gt = rng.standard_normal((B, 1 + k * k, Cout))
+    w = rng.standard_normal((Cout, Cin))
+    pairs = O.select_bases(k, O.RULE_PREFIX, k * k)
+    gx_grid, gw_grid = O.backward_lowrank(xt[:, 1:].reshape(B, k, k, Cin),
+                                          gt[:, 1:].reshape(B, k, k, Cout), w, k, pairs)
+    gx_cls, gw_cls = O.backward_extra_tokens(xt[:, 0], gt[:, 0], w)
+    ex, ew = O.backward_exact(xt, gt, w)
+    assert np.allclose(gw_grid + gw_cls, ew, atol=1e-11)
+    assert np.allclose(gx_cls, ex[:, 0], atol=1e-12)
+    assert np.allclose(gx_grid.reshape(B, k * k, Cin), ex[:, 1:], atol=1e-12)
+    # orientation: one token, one non-zero entry each
+    gxe, gwe = O.backward_extra_tokens(np.eye(1, Cin, 2), np.eye(1, Cout, 1) * 3.0, w)
+    assert gwe[1, 2] == 3.0 and np.count_nonzero(gwe) == 1
+    assert np.allclose(gxe[0], 3.0 * w[1])
+
+
+def test_bias_gradient_is_the_token_sum_and_k_times_the_dc_coefficients():
+    k = 8
+    rng = np.random.default_rng(91)
+    gy = rng.standard_normal((2, 2 * k, k, 5))
+    cls = rng.standard_normal((2, 5))
+    # finite differences of L = <g_y, y + bias> in the bias: dL/db_c = sum of g_y[..., c]
+    want = np.array([gy[..., c].sum() for c in range(5)])
+    assert np.allclose(O.bias_grad(gy), want, atol=1e-12)
+    assert np.allclose(O.bias_grad(gy, cls), want + cls.sum(axis=0), atol=1e-12)
+    # closed form through Eq. 6: B_{0,0} is all ones, so the (0,0) coefficient of a
+    # block is (sum of its tokens) / k
+    for bases in ([(0, 0)], O.select_bases(k, O.RULE_L1, 3)):
+        q = bases.index((0, 0))
+        dc = O.project(gy, k, bases)[:, :, :, q, :]
+        assert np.allclose(k * dc.sum(axis=(0, 1, 2)), want, atol=1e-12)
+    # holds on a zero-extended grid too (the zero tokens add nothing)
+    g7 = rng.standard_normal((1, 7, 7, 3))
+    dc7 = O.project_padded(g7, k, [(0, 0)])[:, :, :, 0, :]
+    assert np.allclose(k * dc7.sum(axis=(0, 1, 2)), O.bias_grad(g7), atol=1e-12)
+
+
+def test_accumulation_over_micro_batches_equals_one_big_batch():
+    k = 4
+    x, gy, w = _tiny(k, 95, B=4)
+    bases = O.select_bases(k, O.RULE_L1, 2)
+    _, whole = O.backward_lowrank(x, gy, w, k, bases)
+    _, first = O.backward_lowrank(x[:2], gy[:2], w, k, bases)
+    _, second = O.backward_lowrank(x[2:], gy[2:], w, k, bases)
+    assert np.allclose(O.accumulate(second, first, 1.0), whole, atol=1e-12)
+    assert np.array_equal(O.accumulate(second, first, 0.0), second)
+    assert np.array_equal(O.accumulate(second), second)
