@@ -173,11 +173,16 @@ int lbp_backward(const void* x, const void* g_y, const void* W,
  * read or write (LBP_ERR_OVERLAP); inputs may be shared.  Knowing that, the
  * library lets the projection kernel of problem i + 1 start on the SMs that the
  * products kernel of problem i has already left instead of waiting for its last
- * tile.  All arguments are checked before anything is enqueued. */
+ * tile.  done_events: NULL, or a host array of n cudaEvent_t handles (as void*,
+ * an entry may be NULL): event i is recorded on `stream` behind the last kernel
+ * of problem i, so that the caller can start what consumes g_W[i] / g_x[i] on
+ * another stream (the data-parallel all-reduce of g_W, the one exchange step
+ * of the path) while the problems that follow still run.  All arguments are
+ * checked before anything is enqueued. */
 int lbp_backward_batch(int n, const void* const* x, const void* const* g_y, const void* const* W,
                        void* const* g_x, void* const* g_W, const lbp_layer* layers,
                        const lbp_basis* set, int r, void* const* ws, const size_t* ws_bytes,
-                       void* stream);
+                       void* const* done_events, void* stream);
 
 /* Eq. 2, exact backpropagation: g_W = g_y^T x over all tokens, g_x = g_y W.
  * This is what all k*k bases give (P P^T = I), computed without transforms.

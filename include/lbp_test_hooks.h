@@ -1,0 +1,34 @@
+/*
+ * lbp_test_hooks.h -- entry points of liblbp that exist for the test suite
+ * only.  They are not part of the library's interface (include/lbp.h) and an
+ * application has no use for them.
+ */
+#ifndef LBP_TEST_HOOKS_H_
+#define LBP_TEST_HOOKS_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Failure injection for the bounded waits of the persistent products kernel
+ * (bf16, r <= 16 path of lbp_backward).  While switched on (per calling
+ * thread), the TMA producer of every products launch issues no load at all.
+ * Nothing is then in flight, the tensor-core issuer and the epilogue warps run
+ * into their wait limits (about a second), the kernel reports LBP_ERR_TIMEOUT
+ * in the status block of the call's workspace, releases its tensor memory and
+ * returns; the outputs of that call are undefined and the context stays
+ * usable.  The paper has no counterpart; this is how the exit path behind
+ * lbp_poll_status is exercised without faulting or hanging a device.
+ * Returns LBP_OK. */
+int lbp_test_stall_products(int on);
+
+/* The library reads its tuning switches (LBP_FUSED, LBP_PAIR, LBP_FUSED_TILES,
+ * LBP_FUSED_VERBOSE) from the environment once, at first use.  This reads them
+ * again, so that one test process can run the same layer through the paths
+ * the switches select.  Returns LBP_OK. */
+int lbp_test_reload_env(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LBP_TEST_HOOKS_H_ */

@@ -14,7 +14,8 @@ from typing import List, Sequence, Tuple
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "liblbp.so")
+# LBP_LIBRARY selects another build of the same library (a diagnostic variant)
+LIB_PATH = os.environ.get("LBP_LIBRARY") or os.path.join(_HERE, "liblbp.so")
 
 LBP_F32, LBP_BF16 = 0, 1
 SEL_L1, SEL_LINF, SEL_PREFIX = 0, 1, 2
@@ -81,7 +82,8 @@ def _lib() -> C.CDLL:
         lib.lbp_backward.restype = i32
         lib.lbp_backward_batch.argtypes = [i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
                                            C.POINTER(vp), C.POINTER(vp), C.POINTER(Layer),
-                                           C.POINTER(Basis), i32, C.POINTER(vp), C.POINTER(sz), vp]
+                                           C.POINTER(Basis), i32, C.POINTER(vp), C.POINTER(sz),
+                                           C.POINTER(vp), vp]
         lib.lbp_backward_batch.restype = i32
         lib.lbp_backward_fullrank.argtypes = [vp, vp, vp, vp, vp, C.POINTER(Layer), vp, sz, vp]
         lib.lbp_backward_fullrank.restype = i32
@@ -90,6 +92,10 @@ def _lib() -> C.CDLL:
         lib.lbp_backward_static.argtypes = [vp, vp, vp, vp, vp, C.POINTER(Layer), C.POINTER(Basis),
                                             i32, vp]
         lib.lbp_backward_static.restype = i32
+        lib.lbp_test_reload_env.argtypes = []
+        lib.lbp_test_reload_env.restype = i32
+        lib.lbp_test_stall_products.argtypes = [i32]
+        lib.lbp_test_stall_products.restype = i32
         lib.lbp_launch_count.argtypes = []
         lib.lbp_launch_count.restype = C.c_longlong
         lib.lbp_set_phase_events.argtypes = [C.POINTER(vp), i32]
@@ -107,7 +113,8 @@ EXPORTED = ("lbp_select_bases", "lbp_basis_matrix", "lbp_flops", "lbp_status_str
             "lbp_expand", "lbp_backward", "lbp_backward_fullrank", "lbp_poll_status",
             "lbp_backward_static", "lbp_launch_count", "lbp_set_phase_events", "lbp_phase_count",
             "lbp_phase_name", "lbp_select_lhe", "lbp_spectrum_workspace_bytes", "lbp_spectrum",
-            "lbp_backward_batch")
+            "lbp_backward_batch", "lbp_test_stall_products",
+            "lbp_test_reload_env")
 
 
 def _check(status: int, where: str) -> None:
@@ -276,10 +283,12 @@ def lbp_backward(x, g_y, W, k: int, bases, *, gw_dtype: torch.dtype = torch.floa
     return g_x, g_W
 
 
-def lbp_backward_batch(xs, g_ys, Ws, k: int, bases, *, g_xs, g_Ws, wss):
+def lbp_backward_batch(xs, g_ys, Ws, k: int, bases, *, g_xs, g_Ws, wss, done_events=None):
     """Algorithm 1 for several independent layers in one call (same k and bases).
     Every argument is a list with one tensor per layer; outputs and workspaces are
-    the caller's and must not overlap anything of another layer."""
+    the caller's and must not overlap anything of another layer.  done_events: an
+    optional list of torch.cuda.Event (or None entries), one per layer, recorded
+    behind that layer's last kernel."""
     n = len(xs)
     lays = (Layer * n)()
     for i in range(n):
@@ -290,9 +299,17 @@ def lbp_backward_batch(xs, g_ys, Ws, k: int, bases, *, g_xs, g_Ws, wss):
     def ptrs(ts, name):
         return (C.c_void_p * n)(*[_dev(t, name) for t in ts])
     sizes = (C.c_size_t * n)(*[w.numel() for w in wss])
+    evs = None
+    if done_events is not None:
+        if len(done_events) != n:
+            raise ValueError("done_events needs one entry per layer")
+        for e in done_events:
+            if e is not None and not e.cuda_event:
+                e.record()          # a torch event has no handle before its first record
+        evs = (C.c_void_p * n)(*[None if e is None else e.cuda_event for e in done_events])
     _check(_lib().lbp_backward_batch(n, ptrs(xs, "x"), ptrs(g_ys, "g_y"), ptrs(Ws, "W"),
                                      ptrs(g_xs, "g_x"), ptrs(g_Ws, "g_W"), lays, _bases(bases),
-                                     len(bases), ptrs(wss, "ws"), sizes, _stream()),
+                                     len(bases), ptrs(wss, "ws"), sizes, evs, _stream()),
            "lbp_backward_batch")
     return g_xs, g_Ws
 
@@ -337,6 +354,18 @@ def lbp_backward_static(x, g_y, W, k: int, bases, *, g_x, g_W):
 def lbp_poll_status(ws: torch.Tensor) -> int:
     """Synchronises the current stream and returns the device status (0 = ok)."""
     return int(_lib().lbp_poll_status(_dev(ws, "ws"), _stream()))
+
+
+def lbp_test_reload_env() -> None:
+    """Test hook: the library reads its LBP_* tuning switches from the environment again."""
+    _check(_lib().lbp_test_reload_env(), "lbp_test_reload_env")
+
+
+def lbp_test_stall_products(on: bool) -> None:
+    """Test hook (include/lbp_test_hooks.h): while on, the products kernel's TMA
+    producers issue nothing, so the call ends in LBP_ERR_TIMEOUT (lbp_poll_status)."""
+    _check(_lib().lbp_test_stall_products(1 if on else 0), "lbp_test_stall_products",
+            "lbp_test_reload_env")
 
 
 # ------------------------------------------------------ measurement hooks ----

@@ -32,15 +32,20 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    """Compile every CUDA source into paper_2309_15275_b200/liblbp.so."""
-    if not force and not _stale():
-        return LIB
+def build_library(force: bool = False, verbose: bool = False, extra_flags=(), out: str | None = None) -> str:
+    """Compile every CUDA source into paper_2309_15275_b200/liblbp.so.
+
+    `extra_flags` (e.g. ["-DLBP_ROLE_TRACE"]) with `out` builds a diagnostic
+    variant into another file; the binding loads it when LBP_LIBRARY names it."""
+    if out is None and not extra_flags:
+        if not force and not _stale():
+            return LIB
+    lib = out or LIB
     objs = []
-    build_dir = os.path.join(HERE, "_build")
+    build_dir = os.path.join(HERE, "_build" if out is None else "_build_variant")
     os.makedirs(build_dir, exist_ok=True)
     common = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+              "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC, *extra_flags]
     if verbose:
         common += ["-Xptxas", "-v"]
     procs = []
@@ -58,9 +63,9 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         failed |= p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    link = [_nvcc(), "-shared", "-o", LIB, *objs, "-lcudart_static", "-ldl", "-lrt", "-lpthread"]
+    link = [_nvcc(), "-shared", "-o", lib, *objs, "-lcudart_static", "-ldl", "-lrt", "-lpthread"]
     subprocess.run(link, check=True)
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":

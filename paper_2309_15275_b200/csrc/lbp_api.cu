@@ -7,6 +7,7 @@
 
 #include "lbp_fused.cuh"
 #include "lbp_internal.h"
+#include "lbp_test_hooks.h"
 
 namespace lbp {
 
@@ -135,10 +136,7 @@ struct Layout {
 
 // The persistent products kernel can be switched off (LBP_FUSED=0) to run the
 // separate product and expansion kernels instead.
-static bool fused_enabled() {
-  const char* e = std::getenv("LBP_FUSED");
-  return !(e != nullptr && e[0] == '0');
-}
+static bool fused_enabled() { return tune_options().fused; }
 
 static Layout plan_layout(const lbp_layer& L, int r) {
   Layout w{};
@@ -292,10 +290,34 @@ static int validate_backward(const void* x, const void* g_y, const void* W, cons
   return LBP_OK;
 }
 
+}  // extern "C"
+
+namespace lbp {
+int validate_backward_call(const void* x, const void* g_y, const void* W, const void* g_x,
+                           const void* g_W, const lbp_layer* layer, const lbp_basis* set, int r,
+                           const void* ws, size_t ws_bytes) {
+  BasisPlan plan;
+  Layout lay;
+  return validate_backward(x, g_y, W, g_x, g_W, layer, set, r, ws, ws_bytes, &plan, &lay);
+}
+}  // namespace lbp
+
+extern "C" {
+
+int lbp_test_reload_env(void) {
+  reload_tune_options();
+  return LBP_OK;
+}
+
+int lbp_test_stall_products(int on) {
+  set_test_stall(on != 0);
+  return LBP_OK;
+}
+
 int lbp_backward_batch(int n, const void* const* x, const void* const* g_y, const void* const* W,
                        void* const* g_x, void* const* g_W, const lbp_layer* layers,
                        const lbp_basis* set, int r, void* const* ws, const size_t* ws_bytes,
-                       void* stream) {
+                       void* const* done_events, void* stream) {
   if (n < 1 || n > 64) return LBP_ERR_SHAPE;
   if (x == nullptr || g_y == nullptr || W == nullptr || g_x == nullptr || g_W == nullptr ||
       layers == nullptr || ws == nullptr || ws_bytes == nullptr)
@@ -341,6 +363,14 @@ int lbp_backward_batch(int n, const void* const* x, const void* const* g_y, cons
     set_projection_defer_wait(i > 0);
     status = lbp_backward(x[i], g_y[i], W[i], g_x[i], g_W[i], &layers[i], set, r, ws[i],
                           ws_bytes[i], stream);
+    if (status == LBP_OK && done_events != nullptr && done_events[i] != nullptr) {
+      const cudaError_t ce = cudaEventRecord(static_cast<cudaEvent_t>(done_events[i]),
+                                             static_cast<cudaStream_t>(stream));
+      if (ce != cudaSuccess) {
+        set_last_cuda_error(ce);
+        status = LBP_ERR_CUDA;
+      }
+    }
   }
   set_projection_defer_wait(false);
   return status;

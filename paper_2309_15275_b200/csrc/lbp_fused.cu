@@ -43,23 +43,23 @@ static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA exceede
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kSlotCols = 256;   // two accumulator slots; tile number t of a CTA uses slot t & 1
 
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-// Optional role timeline (diagnostics): slot 0 kernel start, 2 producer done,
+// Role timeline (diagnostic builds only): slot 0 kernel start, 2 producer done,
 // 3 MMA issuer done, 4 epilogue done, 5 first tile drained.
 __device__ __forceinline__ void trace_mark(const FusedParams& p, int slot, bool first_only = false) {
+#ifdef LBP_ROLE_TRACE
   if (p.trace != nullptr) {
+    unsigned long long now;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
     unsigned long long* t = p.trace + blockIdx.x * 8 + slot;
-    const unsigned long long now = global_ns();
     if (first_only) {
       if (*t == 0) *t = now;
     } else {
       atomicMax(t, now);
     }
   }
+#else
+  (void)p, (void)slot, (void)first_only;
+#endif
 }
 
 // Tile list.  Tiles are numbered with the GW tiles (the larger ones) first and
@@ -183,7 +183,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       const uint64_t keep = ptx::l2_policy_evict_last();
       uint32_t it = 0;
       bool ok = true;
-      for (int ti = 0; ti < my_tiles && ok; ++ti) {
+      for (int ti = 0; ti < my_tiles && ok && !p.test_stall; ++ti) {
         const Tile tl = nth_tile(p, cta, grid, ti);
         const int bn = tl.is_gw ? p.BNw : p.BNx;
         const uint32_t tx = static_cast<uint32_t>(kABytes + bn * BK * 2);
@@ -277,9 +277,14 @@ __global__ void __launch_bounds__(kThreads, 1)
       const uint32_t uses = static_cast<uint32_t>(ti >> 1);
       const uint32_t acc_col = slot * kSlotCols;
       const bool ok = ptx::mbar_wait(&acc_full[slot], uses & 1u, p.status, (4u << 16) | 5u);
-      if (!__all_sync(0xffffffffu, ok)) *abort_flag = 1;
-      named_bar_sync(bar_id, 128);
-      if (*abort_flag) break;
+      // One answer for the whole group: a thread that saw its own wait expire, or
+      // the flag another role raised, takes the other 127 threads with it (read
+      // one by one after the barrier, the flag could split the group, and the
+      // threads left inside the tile would wait on a barrier that never fills).
+      if (named_bar_or(bar_id, 128, !ok || *abort_flag != 0)) {
+        if (etid == 0) *abort_flag = 1;
+        break;
+      }
       ptx::tc_fence_after_sync();
       if (etid == 0 && eg == 0) trace_mark(p, 5, true);
       DrainTile dt;
@@ -308,6 +313,10 @@ __global__ void __launch_bounds__(kThreads, 1)
 }  // namespace fused
 
 // --------------------------------------------------------------- launcher ----
+static thread_local bool g_test_stall = false;
+void set_test_stall(bool on) { g_test_stall = on; }
+bool test_stall() { return g_test_stall; }
+
 bool fused_supported(const lbp_layer& L, const BasisPlan& bp) {
   // the epilogue addresses the tokens of a block with 32-bit element offsets
   const long long block_span = static_cast<long long>(L.k) * L.W * L.Cin;
@@ -386,7 +395,7 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
   p.g_x = static_cast<__nv_bfloat16*>(g_x);
   p.g_W = g_W;
   p.status = status;
-  p.trace = nullptr;
+  p.test_stall = test_stall() ? 1 : 0;
   p.num_kb_x = (L.Cout + BK - 1) / BK;
   p.num_kb_w = p.G * (BM / BK);
   FusedBasis fb;
@@ -503,9 +512,10 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
     if (plan_cache_n < 16) ++plan_cache_n;
   }
   // tuning overrides: LBP_FUSED_TILES="BNw,BNx,splits"
-  if (const char* e = std::getenv("LBP_FUSED_TILES")) {
-    int bw = 0, bx = 0, sp = 0;
-    if (sscanf(e, "%d,%d,%d", &bw, &bx, &sp) == 3 && bw >= 64 && bw <= 256 && bw % 64 == 0 &&
+  if (tune_options().has_tiles) {
+    const int bw = tune_options().tiles_bnw, bx = tune_options().tiles_bnx,
+              sp = tune_options().tiles_splits;
+    if (bw >= 64 && bw <= 256 && bw % 64 == 0 &&
         bx >= 64 && bx <= 256 && bx % 64 == 0 && sp >= 1 && (sp == 1 || sp <= max_splits_by_ws)) {
       p.BNw = bw;
       p.BNx = bx;
@@ -513,8 +523,7 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
       p.gw_splits = (p.num_kb_w + p.kb_per_split_w - 1) / p.kb_per_split_w;
     }
   }
-  if (const char* e = std::getenv("LBP_FUSED_VERBOSE"))
-    if (e[0] == '1')
+  if (tune_options().verbose)
       fprintf(stderr, "lbp products: G=%d BNw=%d BNx=%d gw_splits=%d kb/split=%d\n", p.G, p.BNw, p.BNx,
               p.gw_splits, p.kb_per_split_w);
   p.n_tx = (L.Cin + p.BNx - 1) / p.BNx;
@@ -529,13 +538,10 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
   p.g_x = static_cast<__nv_bfloat16*>(g_x);
   p.g_W = g_W;
   p.status = status;
-  p.trace = nullptr;
-  if (const char* e = std::getenv("LBP_FUSED_TRACE")) {
-    if (e[0] == '1') {
-      p.trace = reinterpret_cast<unsigned long long*>(scratch + lay.trace);
-      LBP_CUDA_TRY(cudaMemsetAsync(p.trace, 0, kFusedTraceBytes, stream));
-    }
-  }
+#ifdef LBP_ROLE_TRACE
+  p.trace = reinterpret_cast<unsigned long long*>(scratch + lay.trace);
+  LBP_CUDA_TRY(cudaMemsetAsync(p.trace, 0, kFusedTraceBytes, stream));
+#endif
 
   // Algorithm 1, steps 1-2: x_hat and g_y_hat, rows padded to 128-row groups
   if (int e = launch_project2(g_y, p.gy_hat, L.Cout, x, p.x_hat, L.Cin, LBP_BF16, L.B, L.H, L.W, bp,

@@ -29,7 +29,12 @@ struct FusedParams {
   __nv_bfloat16* g_x;
   void* g_W;
   uint32_t* status;
-  unsigned long long* trace;              // optional role timeline, 8 slots per CTA (null = off)
+  // failure-injection hook of the test suite (lbp_test_stall_products): the TMA
+  // producers issue no load, so every other role runs into its bounded wait
+  int32_t test_stall;
+#ifdef LBP_ROLE_TRACE
+  unsigned long long* trace;              // role timeline, 8 slots per CTA (null = off)
+#endif
 };
 
 constexpr int kFusedMaxExtra = 2;
@@ -44,12 +49,23 @@ struct FusedBasis {
   uint16_t ex_mv[kFusedMaxExtra];
 };
 
-constexpr size_t kFusedTraceBytes = 256 * 8 * 8;   // last bytes of the scratch region
+// Builds with -DLBP_ROLE_TRACE carry a per-CTA role timeline (diagnostics) in
+// the last bytes of the scratch region; ordinary builds have neither the code
+// nor the bytes.
+#ifdef LBP_ROLE_TRACE
+constexpr size_t kFusedTraceBytes = 256 * 8 * 8;
+#else
+constexpr size_t kFusedTraceBytes = 0;
+#endif
 
 struct FusedLayout {
   size_t x_hat, gy_hat, planes, planes_bytes, trace, total;
   int G, bpt;
 };
+
+// Per-thread switch set by lbp_test_stall_products (test hook).
+void set_test_stall(bool on);
+bool test_stall();
 
 // Called between the projection launch and the products launch (phase events).
 using FusedPhaseHook = int (*)(void* arg, cudaStream_t stream);

@@ -117,6 +117,7 @@ __device__ __forceinline__ void mma_commit_pair(uint64_t* bar) {
 }
 
 __device__ __forceinline__ void trace_mark(const FusedParams& p, int slot, bool first_only = false) {
+#ifdef LBP_ROLE_TRACE
   if (p.trace != nullptr) {
     unsigned long long now;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
@@ -127,6 +128,9 @@ __device__ __forceinline__ void trace_mark(const FusedParams& p, int slot, bool 
       atomicMax(t, now);
     }
   }
+#else
+  (void)p, (void)slot, (void)first_only;
+#endif
 }
 
 // ---- pair-tile list (same snake as the one-CTA kernel, over CTA pairs), taken
@@ -247,7 +251,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       const uint64_t keep = ptx::l2_policy_evict_last();
       uint32_t it = 0;
       bool ok = true;
-      for (int ti = 0; ti < my_tiles && ok; ++ti) {
+      for (int ti = 0; ti < my_tiles && ok && !p.test_stall; ++ti) {
         const PairTile tl = nth_pair_tile(p, pair, pairs, ti);
         const int bn = tl.is_gw ? p.BNw : p.BNx;
         const int half = bn >> 1;
@@ -339,9 +343,14 @@ __global__ void __launch_bounds__(kThreads, 1)
       const int slot = ti & 1;
       const uint32_t uses = static_cast<uint32_t>(ti >> 1);
       const bool ok = ptx::mbar_wait(&acc_full[slot], uses & 1u, p.status, (5u << 16) | 5u);
-      if (!__all_sync(0xffffffffu, ok)) *abort_flag = 1;
-      fused::named_bar_sync(bar_id, 128);
-      if (*abort_flag) break;
+      // One answer for the whole group: a thread that saw its own wait expire, or
+      // the flag another role raised, takes the other 127 threads with it (read
+      // one by one after the barrier, the flag could split the group, and the
+      // threads left inside the tile would wait on a barrier that never fills).
+      if (fused::named_bar_or(bar_id, 128, !ok || *abort_flag != 0)) {
+        if (etid == 0) *abort_flag = 1;
+        break;
+      }
       ptx::tc_fence_after_sync();
       fused::DrainTile dt;
       dt.is_gw = tl.is_gw;
@@ -372,8 +381,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 
 // --------------------------------------------------------------- launcher ----
 bool fused_pair_supported(const lbp_layer& L, int sms) {
-  if (const char* e = std::getenv("LBP_PAIR"))
-    if (e[0] == '0') return false;
+  if (!tune_options().pair) return false;
   return L.Cin >= 128 && sms >= 2 && (sms % 2) == 0;
 }
 
@@ -456,19 +464,17 @@ int launch_fused_pair(const void* x, const void* g_y, const void* W, void* g_W, 
     plan_cache_next = (plan_cache_next + 1) % 16;
     if (plan_cache_n < 16) ++plan_cache_n;
   }
-  if (const char* e = std::getenv("LBP_FUSED_VERBOSE"))
-    if (e[0] == '1')
+  if (tune_options().verbose)
       fprintf(stderr, "lbp products (CTA pairs): G=%d BNw=%d BNx=%d gw_splits=%d kb/split=%d\n", p.G,
               p.BNw, p.BNx, p.gw_splits, p.kb_per_split_w);
-  if (const char* e = std::getenv("LBP_FUSED_TRACE")) {
-    if (e[0] == '1') {
-      p.trace = reinterpret_cast<unsigned long long*>(reinterpret_cast<uint8_t*>(p.x_hat) + lay.trace);
-      LBP_CUDA_TRY(cudaMemsetAsync(p.trace, 0, kFusedTraceBytes, stream));
-    }
-  }
-  if (const char* e = std::getenv("LBP_FUSED_TILES")) {   // tuning override "BNw,BNx,splits"
-    int bw = 0, bx = 0, sp = 0;
-    if (sscanf(e, "%d,%d,%d", &bw, &bx, &sp) == 3 && (bw == 128 || bw == 256) &&
+#ifdef LBP_ROLE_TRACE
+  p.trace = reinterpret_cast<unsigned long long*>(reinterpret_cast<uint8_t*>(p.x_hat) + lay.trace);
+  LBP_CUDA_TRY(cudaMemsetAsync(p.trace, 0, kFusedTraceBytes, stream));
+#endif
+  if (tune_options().has_tiles) {   // tuning override "BNw,BNx,splits"
+    const int bw = tune_options().tiles_bnw, bx = tune_options().tiles_bnx,
+              sp = tune_options().tiles_splits;
+    if ((bw == 128 || bw == 256) &&
         (bx == 128 || bx == 256) && sp >= 1 && (sp == 1 || sp <= max_splits_by_ws)) {
       p.BNw = bw;
       p.BNx = bx;

@@ -29,6 +29,22 @@ __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
+// Barrier over `nthreads` threads that also ORs a predicate over them: every
+// participant gets the same answer, so a decision taken on it (leave the tile
+// loop after an expired wait) cannot split the threads that share the barrier.
+__device__ __forceinline__ bool named_bar_or(int id, int nthreads, bool pred) {
+  uint32_t any;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %3, 0;\n\t"
+      "bar.red.or.pred p, %1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(any)
+      : "r"(id), "r"(nthreads), "r"(static_cast<uint32_t>(pred))
+      : "memory");
+  return any != 0;
+}
+
 __device__ __forceinline__ int blocks_in_group(const FusedParams& p, int g) {
   const int left = p.nb - g * p.bpt;
   return left < p.bpt ? left : p.bpt;

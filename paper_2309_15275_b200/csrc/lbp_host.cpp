@@ -106,6 +106,29 @@ static bool prefix_less(const PairKey& a, const PairKey& b) {
 
 using namespace lbp;
 
+namespace lbp {
+static TuneOptions g_tune;
+static bool g_tune_loaded = false;
+void reload_tune_options() {
+  TuneOptions t{};
+  const char* e = std::getenv("LBP_FUSED");
+  t.fused = !(e != nullptr && e[0] == '0');
+  e = std::getenv("LBP_PAIR");
+  t.pair = !(e != nullptr && e[0] == '0');
+  e = std::getenv("LBP_FUSED_VERBOSE");
+  t.verbose = e != nullptr && e[0] == '1';
+  e = std::getenv("LBP_FUSED_TILES");
+  t.has_tiles = e != nullptr &&
+                std::sscanf(e, "%d,%d,%d", &t.tiles_bnw, &t.tiles_bnx, &t.tiles_splits) == 3;
+  g_tune = t;
+  g_tune_loaded = true;
+}
+const TuneOptions& tune_options() {
+  if (!g_tune_loaded) reload_tune_options();
+  return g_tune;
+}
+}  // namespace lbp
+
 extern "C" {
 
 int lbp_select_bases(int k, int rule, int param, lbp_basis* out, int cap, int* r_out) {

@@ -130,4 +130,23 @@ int launch_splitk_reduce(const float* planes, void* D, long long mn, int splits,
 
 int check_device_arch();
 
+// Tuning switches, read from the environment once (first use):
+//   LBP_FUSED=0          separate product and expansion kernels instead of the
+//                        persistent products kernel
+//   LBP_PAIR=0           one-CTA products kernel also on wide layers
+//   LBP_FUSED_TILES=a,b,c  column tiles of the two products and K slices of g_W
+//   LBP_FUSED_VERBOSE=1  print the chosen tile plan
+struct TuneOptions {
+  bool fused, pair, verbose, has_tiles;
+  int tiles_bnw, tiles_bnx, tiles_splits;
+};
+const TuneOptions& tune_options();
+void reload_tune_options();   // test hook: read the environment again
+
+// Every host-side check of one lbp_backward call (pointers, layer, basis list,
+// alignment, workspace size); nothing is enqueued.  Returns an lbp_status.
+int validate_backward_call(const void* x, const void* g_y, const void* W, const void* g_x,
+                           const void* g_W, const lbp_layer* layer, const lbp_basis* set, int r,
+                           const void* ws, size_t ws_bytes);
+
 }  // namespace lbp

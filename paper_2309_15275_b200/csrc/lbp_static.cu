@@ -18,6 +18,8 @@
 // the kernels receive.
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "lbp.h"
 #include "lbp_internal.h"
 
@@ -28,7 +30,7 @@ constexpr size_t kStaticScratchBytes = LBP_STATIC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 constexpr int kMaxDevices = 64;
-void* g_scratch_addr[kMaxDevices] = {};
+std::atomic<void*> g_scratch_addr[kMaxDevices] = {};
 
 // Device address of the scratch array on the current device (looked up on the
 // first call per device; a query, not an allocation).
@@ -36,12 +38,13 @@ int static_scratch_address(void** out) {
   int dev = 0;
   LBP_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices) return LBP_ERR_ARCH;
-  if (g_scratch_addr[dev] == nullptr) {
-    void* ptr = nullptr;
+  void* ptr = g_scratch_addr[dev].load(std::memory_order_acquire);
+  if (ptr == nullptr) {
+    // two threads may both look it up: they get the same address
     LBP_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
-    g_scratch_addr[dev] = ptr;
+    g_scratch_addr[dev].store(ptr, std::memory_order_release);
   }
-  *out = g_scratch_addr[dev];
+  *out = ptr;
   return LBP_OK;
 }
 
@@ -51,11 +54,16 @@ extern "C" int lbp_backward_static(const void* x, const void* g_y, const void* W
                                    void* g_W, const lbp_layer* layer, const lbp_basis* set, int r,
                                    void* stream) {
   if (layer == nullptr) return LBP_ERR_NULL;
-  // 0 means an invalid layer or rank: lbp_backward below names the exact error
+  // 0 means an invalid layer or rank: the validation below names the exact error
   const size_t need = lbp_workspace_bytes(layer, r);
   if (need > kStaticScratchBytes) return LBP_ERR_WORKSPACE;  // beyond the built-in scratch
+  if (int e = lbp::check_device_arch()) return e;
   void* scratch = nullptr;
   if (int e = static_scratch_address(&scratch)) return e;
+  // every argument check of lbp_backward, before anything is enqueued
+  if (int e = lbp::validate_backward_call(x, g_y, W, g_x, g_W, layer, set, r, scratch,
+                                          kStaticScratchBytes))
+    return e;
   // The array keeps what the previous call left in it.  Only the status block
   // must start clean (a stale report would be read as this call's); x_hat,
   // g_y_hat and the partial sums are fully rewritten before they are read.

@@ -3,8 +3,18 @@
 Every comparison is on the same seeded inputs, already rounded to the run
 dtype.  Bars: relative Frobenius error <= 1e-5 for fp32 data, <= 2e-2 for bf16
 data with fp32 accumulation; basis lists bit-exact (checked on the CPU suite).
+
+Beside the global bar every backward comparison has a local one, so that a
+wrong patch cannot hide in the norm of a large tensor: the largest relative
+Frobenius error over the k x k token blocks of g_x and over 128 x 128 pieces of
+g_W.  For bf16 data the error is rounding noise of x_hat, g_y_hat and the
+outputs to 8 mantissa bits (about 2^-9 per element, 2.4e-3 observed in the
+norm of whole tensors); a block holds thousands of such elements, so its norm
+ratio sits near the same figure, and the local bar is 1e-2, four times that.
+A misplaced or dropped coefficient changes a block by the order of its norm.
 """
 import functools
+import os
 
 import numpy as np
 import pytest
@@ -17,6 +27,7 @@ from oracle import lbp_oracle as O
 pytestmark = pytest.mark.gpu
 
 TOL = {torch.float32: 1e-5, torch.bfloat16: 2e-2}
+LOCAL_TOL = {torch.float32: 1e-5, torch.bfloat16: 1e-2}
 
 
 @pytest.fixture(scope="module")
@@ -36,6 +47,14 @@ def rel(got, want):
 
 def ok_status(ws):
     assert lbp.lbp_poll_status(ws) == 0
+
+
+def coef_block_rel(got, want):
+    """Largest relative error over the blocks of a coefficient tensor (B,Hb,Wb,r,C)."""
+    d = f64(got) - want
+    num = np.sqrt(np.sum(d * d, axis=(3, 4)))
+    den = np.sqrt(np.sum(want * want, axis=(3, 4)))
+    return float(np.max(np.where(den > 0, num / np.where(den > 0, den, 1.0), num)))
 
 
 @functools.lru_cache(maxsize=2)
@@ -59,10 +78,13 @@ def test_project_expand_prefix_sets(dev, dtype, k, ranks):
         want = O.project(f64(t), k, bases)
         assert got.shape == want.shape
         assert rel(got, want) <= TOL[dtype], (k, r)
+        assert coef_block_rel(got, want) <= LOCAL_TOL[dtype], (k, r)
         th = torch.from_numpy(want).to(dtype)
         back = lbp.lbp_expand(th.to(dev), k, bases, ws=ws)
         ok_status(ws)
-        assert rel(back, O.expand(f64(th), k, bases)) <= TOL[dtype], (k, r)
+        want_back = O.expand(f64(th), k, bases)
+        assert rel(back, want_back) <= TOL[dtype], (k, r)
+        assert O.block_rel_fro(f64(back), want_back, k) <= LOCAL_TOL[dtype], (k, r)
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
@@ -134,12 +156,17 @@ def _run_backward(dev, case, r, batch=None, fullrank_entry=False, bases=None, id
     return (x, gy, w), bases, gx, gw
 
 
+def _assert_parity(gx, gw, ox, ow, k, dtype, what):
+    assert rel(gx, ox) <= TOL[dtype], (what, "g_x")
+    assert rel(gw, ow) <= TOL[dtype], (what, "g_W")
+    assert O.block_rel_fro(f64(gx), ox, k) <= LOCAL_TOL[dtype], (what, "g_x, worst block")
+    assert O.tile_rel_fro(f64(gw), ow, 128) <= LOCAL_TOL[dtype], (what, "g_W, worst 128 x 128 piece")
+
+
 def _check_lowrank(dev, case, r, batch=None, bases=None):
     (x, gy, w), bases, gx, gw = _run_backward(dev, case, r, batch, bases=bases)
     ox, ow = O.backward_lowrank(f64(x), f64(gy), f64(w), case.k, bases)
-    tol = TOL[x.dtype]
-    assert rel(gx, ox) <= tol, (case.name, r, "g_x")
-    assert rel(gw, ow) <= tol, (case.name, r, "g_W")
+    _assert_parity(gx, gw, ox, ow, case.k, x.dtype, (case.name, r))
 
 
 def test_config1_fp32(dev):
@@ -169,11 +196,26 @@ def test_config2_efficientformer_full_size(dev, idx):
     _check_lowrank(dev, synth.config_cases(2)[idx], 8)
 
 
-@pytest.mark.parametrize("idx,ranks", [(0, (8,)), (1, (2, 4, 8, 16)), (2, (8, 16)), (3, (2, 8))])
-def test_config3_vitb_full_size(dev, idx, ranks):
+@pytest.mark.parametrize("idx", [0, 1, 2, 3])
+def test_config3_vitb_full_size(dev, idx):
+    # every layer of the block at every rank of the configuration
     case = synth.config_cases(3)[idx]
-    for r in ranks:
+    for r in (2, 4, 8, 16):
         _check_lowrank(dev, case, r)
+
+
+@pytest.mark.parametrize("switch", ["LBP_PAIR", "LBP_FUSED"])
+def test_config3_through_the_switched_paths(dev, switch):
+    # LBP_PAIR=0: the one-CTA products kernel on wide layers; LBP_FUSED=0: separate
+    # product and expansion kernels.  Same bars as the default path.
+    os.environ[switch] = "0"
+    lbp.lbp_test_reload_env()
+    try:
+        for idx in (1, 2):
+            _check_lowrank(dev, synth.config_cases(3)[idx], 8)
+    finally:
+        del os.environ[switch]
+        lbp.lbp_test_reload_env()
 
 
 @pytest.mark.parametrize("idx", [0, 1])
@@ -214,11 +256,22 @@ def test_bf16_full_rank_is_exact_bp(dev):
         assert rel(gx, ex) <= 2e-2 and rel(gw, ew) <= 2e-2
 
 
-@pytest.mark.parametrize("idx,ranks", [(0, (1, 4, 7, 16)), (1, (1, 8, 21, 36)), (2, (1, 10, 36, 100))])
+# ranks chosen so that every expansion variant of the products kernel (cores of
+# 1, 2, 4 and 8 coefficients per side, the 4 x 4 core plus one or two extra
+# bases at r = 14..16), the generic path (r > 16) and the full-rank mode run at
+# full size
+@pytest.mark.parametrize("idx,ranks", [(0, (1, 2, 4, 7, 12, 16)),
+                                       (1, (1, 2, 3, 5, 8, 11, 12, 13, 14, 15, 21, 36, 64)),
+                                       (2, (1, 3, 5, 10, 14, 16, 36, 100, 256))])
 def test_config5_sweep_full_size(dev, idx, ranks):
     case = synth.config_cases(5)[idx]
     for r in ranks:
-        _check_lowrank(dev, case, r)
+        if r == case.k * case.k:
+            (x, gy, w), _, gx, gw = _run_backward(dev, case, r)
+            ex, ew = O.backward_exact(f64(x), f64(gy), f64(w))
+            _assert_parity(gx, gw, ex, ew, case.k, x.dtype, (case.name, "full rank"))
+        else:
+            _check_lowrank(dev, case, r)
 
 
 def test_outputs_do_not_depend_on_basis_order(dev):
@@ -228,7 +281,12 @@ def test_outputs_do_not_depend_on_basis_order(dev):
     perm = [bases[i] for i in (3, 0, 5, 1, 4, 2)]
     a = lbp.lbp_backward(x.to(dev), gy.to(dev), w.to(dev), 8, bases)
     b = lbp.lbp_backward(x.to(dev), gy.to(dev), w.to(dev), 8, perm)
-    assert rel(a[0], f64(b[0])) <= 1e-2 and rel(a[1], f64(b[1])) <= 1e-2
+    ox, ow = O.backward_lowrank(f64(x), f64(gy), f64(w), 8, bases)
+    for got in (a, b):
+        _assert_parity(got[0], got[1], ox, ow, 8, x.dtype, "order")
+    # the order only permutes the rows of x_hat / g_y_hat: the sums of g_W are taken
+    # in another order (fp32), g_x sees the same arithmetic
+    assert rel(b[1], f64(a[1])) <= 1e-5 and rel(b[0], f64(a[0])) <= 1e-3
 
 
 def test_repeated_calls_are_deterministic(dev):
@@ -261,9 +319,12 @@ def test_spectrum_matches_oracle(dev, dtype, k):
     want = O.spectrum(f64(t), k)
     got = e.cpu().numpy()
     assert got.shape == (k, k)
-    # energies are sums of squares of coefficients held in `dtype`
-    tol = 1e-5 if dtype == torch.float32 else 2e-2
-    assert np.max(np.abs(got - want) / want.max()) <= tol
+    # Every energy on its own, so that the weak responses (the ones a selection
+    # ranks) are held to the same bar as the DC term.  fp32 data: coefficients and
+    # sums in fp32.  bf16 data: the +-1 products of bf16 values are exact, sums in
+    # fp32 / fp64, nothing is rounded to bf16 on the way.
+    tol = 1e-5 if dtype == torch.float32 else 1e-4
+    assert np.max(np.abs(got - want) / want) <= tol
     assert abs(got.sum() - np.sum(f64(t) ** 2)) <= tol * np.sum(f64(t) ** 2)   # Parseval
     # the selection is taken on the host from the energies: same list wherever
     # the oracle's energies are separated by more than the tolerance
@@ -271,7 +332,7 @@ def test_spectrum_matches_oracle(dev, dtype, k):
         sel = lbp.lbp_select_lhe(got, k, r)
         ref = O.select_lhe(want, k, r)
         srt = np.sort(want.ravel())[::-1]
-        if r < k * k and (srt[r - 1] - srt[r]) > 4 * tol * want.max():
+        if r < k * k and (srt[r - 1] - srt[r]) > 4 * tol * srt[r - 1]:
             assert set(sel) == set(ref)
         assert sel == O.select_lhe(got, k, r)
     # second call into the same output: overwritten, not accumulated
@@ -290,7 +351,7 @@ def test_spectrum_full_size_layer_and_lhe_backward(dev):
     # sampled check against the oracle: 8 images
     want = O.spectrum(f64(gy[:8]), k)
     got8 = lbp.lbp_spectrum(gy[:8].contiguous().to(dev), k).cpu().numpy()
-    assert np.max(np.abs(got8 - want)) <= 2e-2 * want.max()
+    assert np.max(np.abs(got8 - want) / want) <= 1e-4
     bases = lbp.lbp_select_lhe(e, k, 8)
     assert len(set(bases)) == 8
     xs, gs = x[:4].contiguous(), gy[:4].contiguous()

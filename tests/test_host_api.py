@@ -20,7 +20,8 @@ def _built():
 
 
 def test_library_exports_every_declared_symbol():
-    header = open(os.path.join(ROOT, "include", "lbp.h")).read()
+    inc = os.path.join(ROOT, "include")
+    header = "".join(open(os.path.join(inc, f)).read() for f in sorted(os.listdir(inc)) if f.endswith(".h"))
     declared = set(re.findall(r"^(?:int|size_t|double|long long|const char\*)\s+(lbp_[a-z_]+)\s*\(", header, re.M))
     assert declared == set(lbp.EXPORTED)
     lib = ctypes.CDLL(lbp.LIB_PATH)
@@ -141,7 +142,7 @@ def test_batch_arguments_are_checked_on_the_host_before_any_device_call():
     def call(x, gy, w, gx, gw, ws, sizes=None):
         sz = (ctypes.c_size_t * n)(*(sizes or need))
         return lib.lbp_backward_batch(n, arr(x), arr(gy), arr(w), arr(gx), arr(gw), lays,
-                                      b._bases(bases), r, arr(ws), sz, None)
+                                      b._bases(bases), r, arr(ws), sz, None, None)
 
     x = [base, base + 64 * MB]
     gy = [base + 8 * MB, base + 72 * MB]
@@ -161,5 +162,5 @@ def test_batch_arguments_are_checked_on_the_host_before_any_device_call():
     assert call(x, gy, w, [gx[0], gx[1] + 2], gw, ws) == 6          # misaligned pointer
     assert call(x, gy, w, [gx[0], None], gw, ws) == 1               # null pointer
     assert lib.lbp_backward_batch(0, arr(x), arr(gy), arr(w), arr(gx), arr(gw), lays,
-                                  b._bases(bases), r, arr(ws), (ctypes.c_size_t * n)(*need), None) == 2
+                                  b._bases(bases), r, arr(ws), (ctypes.c_size_t * n)(*need), None, None) == 2
     assert "overlap" in lbp.lbp_status_string(12)
