@@ -25,7 +25,6 @@ import os
 import statistics
 import subprocess
 import sys
-import threading
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -59,59 +58,76 @@ NCU_TRAFFIC_PER_STEP = {"wht_project_mma_kernel": None, "lbp_products_pair_kerne
 
 
 # ------------------------------------------------------------------ clocks ----
-class ClockSampler:
-    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+_SAMPLER_CODE = r"""
+import sys, time
+import pynvml as n
+n.nvmlInit()
+h = n.nvmlDeviceGetHandleByIndex(int(sys.argv[1]))
+print("max", n.nvmlDeviceGetMaxClockInfo(h, n.NVML_CLOCK_SM), flush=True)
+end = time.time() + 120.0
+while time.time() < end:
+    mhz = n.nvmlDeviceGetClockInfo(h, n.NVML_CLOCK_SM)
+    try:
+        mask = n.nvmlDeviceGetCurrentClocksEventReasons(h)
+    except Exception:
+        mask = n.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+    print(repr(time.time()), mhz, mask, flush=True)
+"""
 
-    def __init__(self, index: int, period_s: float = 0.0005):
-        self.index, self.period = index, period_s
-        self.samples, self.reasons = [], set()
-        self.max_mhz = None
-        self._stop = threading.Event()
-        self._thread = None
-        self._nvml = None
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region
+    runs.  The sampling loop lives in a child process (started before the timed
+    region, no GPU context of its own): a thread of this process would share the
+    interpreter lock with the launching loop and hardly ever run."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap"}
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
 
     def start(self):
         try:
-            import pynvml
-            pynvml.nvmlInit()
-            self._nvml = pynvml
-            self._h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
-            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+            self.proc = subprocess.Popen([sys.executable, "-c", _SAMPLER_CODE, str(self.index)],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.max_line = self.proc.stdout.readline()      # the child is up and sampling
         except Exception:
-            self._nvml = None
-            return
-        self._thread = threading.Thread(target=self._run, daemon=True)
-        self._thread.start()
+            self.proc = None
 
-    def _run(self):
-        n = self._nvml
-        names = {
-            getattr(n, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
-            getattr(n, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
-            getattr(n, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
-            getattr(n, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
-        }
-        while not self._stop.is_set():
-            try:
-                self.samples.append(n.nvmlDeviceGetClockInfo(self._h, n.NVML_CLOCK_SM))
+    def stop(self, t_begin: float, t_end: float):
+        """Summary of the samples taken between the two time.time() stamps."""
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        out = self.proc.stdout.read()
+        self.proc.wait()
+        max_mhz = None
+        try:
+            max_mhz = int(self.max_line.split()[1])
+        except Exception:
+            pass
+        rows = []
+        for ln in out.splitlines():
+            f = ln.split()
+            if len(f) == 3:
                 try:
-                    mask = n.nvmlDeviceGetCurrentClocksEventReasons(self._h)
-                except Exception:
-                    mask = n.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
-                for bit, name in names.items():
-                    if mask & bit:
-                        self.reasons.add(name)
-            except Exception:
-                pass
-            time.sleep(self.period)
-
-    def stop(self):
-        self._stop.set()
-        if self._thread is not None:
-            self._thread.join(timeout=2)
-        med = statistics.median(self.samples) if self.samples else None
-        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+                    rows.append((float(f[0]), int(f[1]), int(f[2])))
+                except ValueError:
+                    pass
+        inside = [r for r in rows if t_begin <= r[0] <= t_end]
+        if not inside and rows:     # a region shorter than one sampling period: the nearest sample
+            mid = 0.5 * (t_begin + t_end)
+            inside = [min(rows, key=lambda r: abs(r[0] - mid))]
+        reasons = set()
+        for _, _, mask in inside:
+            for bit, name in self.REASONS.items():
+                if mask & bit:
+                    reasons.add(name)
+        med = statistics.median([r[1] for r in inside]) if inside else None
+        return {"sm_mhz": med, "sm_max_mhz": max_mhz, "reasons": sorted(reasons),
+                "samples": len(inside), "sampling": "NVML from a child process, back to back"}
 
 
 # ------------------------------------------------------------- cpu oracle ----
@@ -304,16 +320,17 @@ def run_gpu(args):
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-        time.sleep(0.002)
     launches0 = lbp.lbp_launch_count()
     t_beg, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    wall0 = time.time()
     t_beg.record()
     for _ in range(steps):
         step()
     t_end.record()
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    wall1 = time.time()
+    clocks = sampler.stop(wall0, wall1) if rank == 0 else None
     launches = lbp.lbp_launch_count() - launches0
     ms_total = t_beg.elapsed_time(t_end)
     for L in layers:

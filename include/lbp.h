@@ -20,10 +20,15 @@
  *  - Layouts are dense, channels-last raster:
  *        x   (B, H, W, Cin)     g_y (B, H, W, Cout)     g_x (B, H, W, Cin)
  *        W, g_W (Cout, Cin) row-major (w in R^{Cy x Cx} of Eq. 1)
- *        t_hat (B, H/k, W/k, r, C): coefficient q of a block follows the order
- *        of the basis list.
+ *        t_hat (B, ceil(H/k), ceil(W/k), r, C): coefficient q of a block follows
+ *        the order of the basis list.
  *    Tokens are grouped into non-overlapping, origin-aligned k x k blocks of
- *    the (H, W) grid; H and W must be multiples of k.
+ *    the (H, W) grid.  The paper does not say what happens to a grid whose
+ *    sides are not multiples of the transform order (its own 7 x 7 maps of
+ *    Sec. 3.3 and Table 5); here such a grid is extended with zero tokens at
+ *    its high end (bottom rows, right columns) to the next multiples of k: a
+ *    side of n tokens has ceil(n / k) blocks, the zero tokens are never read
+ *    from or written to memory, and g_x is produced for the real tokens only.
  *  - Bases are orthonormal: the +-1 Walsh bases of Eq. 6-7 are scaled by 1/k
  *    in the projection and by 1/k in the reverse projection, so that all k*k
  *    bases reproduce exact backpropagation (Sec. 3, completeness).
@@ -51,7 +56,7 @@ extern "C" {
 typedef enum {
   LBP_OK = 0,
   LBP_ERR_NULL = 1,       /* a required pointer is NULL                         */
-  LBP_ERR_SHAPE = 2,      /* a dimension <= 0, or H % k != 0, or W % k != 0      */
+  LBP_ERR_SHAPE = 2,      /* a dimension or count out of range                  */
   LBP_ERR_BLOCK = 3,      /* k not in {4, 8, 16}                                */
   LBP_ERR_BASIS = 4,      /* r < 1, r > k*k, index outside [0,k), duplicate pair */
   LBP_ERR_DTYPE = 5,      /* unknown dtype, or a combination not supported      */
@@ -127,7 +132,7 @@ size_t lbp_status_bytes(void);
 
 /* Eq. 6 per block:  t_hat[b,bh,bw,q,c] = (1/k) sum_{u,v} wal_iq[u] wal_jq[v]
  *                                         t[b, bh*k+u, bw*k+v, c].
- * t (B,H,W,C) -> t_hat (B,H/k,W/k,r,C), both of `dtype`; fp32 accumulation,
+ * t (B,H,W,C) -> t_hat (B,ceil(H/k),ceil(W/k),r,C), both of `dtype`; fp32 accumulation,
  * one rounding to the output type.  ws: >= lbp_status_bytes(). */
 int lbp_project(const void* t, void* t_hat, int B, int H, int W, int C, int k,
                 const lbp_basis* set, int r, int dtype,
@@ -149,7 +154,7 @@ int lbp_spectrum(const void* t, double* energy, int B, int H, int W, int C, int 
 
 /* Eq. 7 per block:  t[b,bh*k+u,bw*k+v,c] = (1/k) sum_q wal_iq[u] wal_jq[v]
  *                                          t_hat[b,bh,bw,q,c].
- * t_hat (B,H/k,W/k,r,C) -> t (B,H,W,C), both of `dtype`. */
+ * t_hat (B,ceil(H/k),ceil(W/k),r,C) -> t (B,H,W,C), both of `dtype`. */
 int lbp_expand(const void* t_hat, void* t, int B, int H, int W, int C, int k,
                const lbp_basis* set, int r, int dtype,
                void* ws, size_t ws_bytes, void* stream);
@@ -183,6 +188,53 @@ int lbp_backward_batch(int n, const void* const* x, const void* const* g_y, cons
                        void* const* g_x, void* const* g_W, const lbp_layer* layers,
                        const lbp_basis* set, int r, void* const* ws, const size_t* ws_bytes,
                        void* const* done_events, void* stream);
+
+/* What a linear layer of a real ViT needs around Algorithm 1 and the paper
+ * leaves out (Eq. 1 has no bias; Sec. 3 knows only the tokens of the grid).
+ * All pointers are device pointers; the struct itself is read on the host. */
+typedef struct {
+  /* g_W <- beta * g_W + (g_W of this call); 0 overwrites.  beta = 1 adds a
+   * micro-batch to an accumulated gradient.  g_bias follows the same rule. */
+  float beta;
+  /* NULL, or fp32[Cout]: gradient of a bias added to y, the sum of g_y over all
+   * tokens (grid and extra).  With the basis (0,0) in the list this is k times
+   * the sum of the DC coefficients of g_y_hat (exact in exact arithmetic: that
+   * basis is the block sum scaled by 1/k); otherwise g_y is read once more. */
+  void* g_bias;
+  /* Tokens that are not part of the grid (a class token per image): the method
+   * says nothing about them, so they take Eq. 2 exactly: g_x_extra = g_y_extra W
+   * and g_y_extra^T x_extra is added to g_W.  n_extra = 0: none.
+   * x_extra (n_extra, Cin), gy_extra (n_extra, Cout), gx_extra (n_extra, Cin),
+   * of the layer's dtype. */
+  int32_t n_extra;
+  const void* x_extra;
+  const void* gy_extra;
+  void* gx_extra;
+} lbp_extras;
+
+/* Scratch for lbp_backward_ex (>= lbp_workspace_bytes; 0 = invalid arguments). */
+size_t lbp_workspace_bytes_ex(const lbp_layer* layer, int r, const lbp_extras* ex);
+
+/* Algorithm 1 with the parts above.  Exactly one of x and x_hat is given:
+ *  - x (B,H,W,Cin): as lbp_backward;
+ *  - x_hat (B,ceil(H/k),ceil(W/k),r,Cin) = p(x), the output of lbp_project with the
+ *    same k and basis list (Eq. 3), taken at forward time so that only r / k^2
+ *    of the activation is kept until the backward pass; Algorithm 1 then starts
+ *    at its second step (g_y_hat = p(g_y)).  The result equals lbp_backward on
+ *    x up to the rounding of x_hat to `dtype` that both take.
+ * ex may be NULL (then this is lbp_backward / lbp_backward_projected).
+ * ws: >= lbp_workspace_bytes_ex(layer, r, ex). */
+int lbp_backward_ex(const void* x, const void* x_hat, const void* g_y, const void* W,
+                    void* g_x, void* g_W, const lbp_layer* layer,
+                    const lbp_basis* set, int r, const lbp_extras* ex,
+                    void* ws, size_t ws_bytes, void* stream);
+
+/* Algorithm 1 from its second step on (Eq. 3 applied to x beforehand):
+ * lbp_backward_ex with x = NULL and no extras.  ws: >= lbp_workspace_bytes. */
+int lbp_backward_projected(const void* x_hat, const void* g_y, const void* W,
+                           void* g_x, void* g_W, const lbp_layer* layer,
+                           const lbp_basis* set, int r,
+                           void* ws, size_t ws_bytes, void* stream);
 
 /* Eq. 2, exact backpropagation: g_W = g_y^T x over all tokens, g_x = g_y W.
  * This is what all k*k bases give (P P^T = I), computed without transforms.

@@ -6,6 +6,8 @@
 #ifndef LBP_TEST_HOOKS_H_
 #define LBP_TEST_HOOKS_H_
 
+#include <stdint.h>
+
 #ifdef __cplusplus
 extern "C" {
 #endif
@@ -21,6 +23,16 @@ extern "C" {
  * lbp_poll_status is exercised without faulting or hanging a device.
  * Returns LBP_OK. */
 int lbp_test_stall_products(int on);
+
+/* Host-side tile plan of the persistent products kernel for a layer of Cin x
+ * Cout channels whose low-rank rows fill G groups of 128 rows (bpt blocks per
+ * group, order k), on `units` CTAs (pair = 0) or CTA pairs (pair = 1).
+ * out6 = {BNw, BNx, K slices of g_W, k-blocks per slice, listed, tiles listed};
+ * first: 161 entries, ids: 1536 entries: unit u works, in this order, on the
+ * tiles ids[first[u]] .. ids[first[u+1]-1]; ids below (row tiles of g_W) *
+ * (column tiles) * slices are GW tiles, the others GX tiles.  No device needed. */
+int lbp_test_tile_plan(int Cin, int Cout, int G, int bpt, int k, int units, int pair,
+                       int max_splits, int epi_kind, int32_t* out6, uint16_t* first, uint16_t* ids);
 
 /* The library reads its tuning switches (LBP_FUSED, LBP_PAIR, LBP_FUSED_TILES,
  * LBP_FUSED_VERBOSE) from the environment once, at first use.  This reads them

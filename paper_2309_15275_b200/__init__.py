@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     lbp_status_string, lbp_workspace_bytes, lbp_launch_count, lbp_phase_count, lbp_phase_name,
     lbp_set_phase_events, lbp_backward_static, STATIC_SCRATCH_BYTES,
     lbp_select_lhe, lbp_spectrum, lbp_spectrum_workspace_bytes, lbp_backward_batch,
-    lbp_test_stall_products, lbp_test_reload_env,
+    lbp_test_stall_products, lbp_test_reload_env, lbp_test_tile_plan,
+    lbp_backward_ex, lbp_backward_projected, lbp_workspace_bytes_ex,
 )
 from .autograd import LbpLinear, LbpLinearFunction  # noqa: F401,E402

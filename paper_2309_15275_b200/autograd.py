@@ -2,8 +2,9 @@
 Algorithm 1 (low-rank backpropagation on the selected Walsh-Hadamard bases).
 
 Only the backward pass is the library's: the forward product `y = x W^T` is a
-plain matrix product and is left to torch.  The layer has no bias (the paper's
-Eq. 1) and expects the token grid explicit: x of shape (B, H, W, Cin).
+plain matrix product and is left to torch.  The layer expects the token grid
+explicit: x of shape (B, H, W, Cin); the bias (absent from the paper's Eq. 1) is
+optional.
 """
 from __future__ import annotations
 
@@ -15,39 +16,59 @@ from . import binding as _b
 
 
 class LbpLinearFunction(torch.autograd.Function):
-    """y = x W^T;  backward: (g_x, g_W) = lbp_backward(x, g_y, W, k, bases)."""
+    """y = x W^T (+ b);  backward: Algorithm 1 on the selected bases.
+
+    With `save_projected` the forward pass keeps x_hat = p(x) (Eq. 3) instead of
+    x: r / k^2 of the activation's elements stay alive until the backward pass,
+    which then starts at the second step of Algorithm 1."""
 
     @staticmethod
-    def forward(ctx, x: torch.Tensor, weight: torch.Tensor, k: int,
-                bases: Sequence[Tuple[int, int]]):
+    def forward(ctx, x: torch.Tensor, weight: torch.Tensor, bias, k: int,
+                bases: Sequence[Tuple[int, int]], save_projected: bool):
         if x.dim() != 4:
             raise ValueError("x must be (B, H, W, Cin)")
-        ctx.save_for_backward(x, weight)
         ctx.k, ctx.bases = int(k), [tuple(p) for p in bases]
-        return torch.matmul(x, weight.t())
+        ctx.projected = bool(save_projected) and x.is_cuda
+        ctx.has_bias = bias is not None
+        if ctx.projected:
+            ctx.save_for_backward(_b.lbp_project(x.contiguous(), ctx.k, ctx.bases), weight)
+        else:
+            ctx.save_for_backward(x, weight)
+        y = torch.matmul(x, weight.t())
+        return y if bias is None else y + bias
 
     @staticmethod
     def backward(ctx, g_y: torch.Tensor):
-        x, weight = ctx.saved_tensors
-        g_x, g_W = _b.lbp_backward(x.contiguous(), g_y.contiguous(), weight.contiguous(), ctx.k,
-                                   ctx.bases, gw_dtype=weight.dtype)
-        return g_x, g_W, None, None
+        saved, weight = ctx.saved_tensors
+        g_y = g_y.contiguous()
+        g_b = (torch.empty(weight.shape[0], dtype=torch.float32, device=g_y.device)
+               if ctx.has_bias else None)
+        kw = {"x_hat": saved} if ctx.projected else {}
+        g_x, g_W = _b.lbp_backward_ex(None if ctx.projected else saved.contiguous(), g_y,
+                                      weight.contiguous(), ctx.k, ctx.bases, g_bias=g_b,
+                                      gw_dtype=weight.dtype, **kw)
+        return g_x, g_W, (None if g_b is None else g_b.to(weight.dtype)), None, None, None
 
 
 class LbpLinear(torch.nn.Module):
-    """Bias-free linear layer over a (B, H, W, C) token grid with LBP-WHT backward.
+    """Linear layer over a (B, H, W, C) token grid with LBP-WHT backward.
 
     `bases` is an ordered list of 0-based (i, j) sequency pairs, e.g. from
     `lbp_select_bases(k, SEL_L1, m)` (Eq. 8) or `lbp_select_lhe` (Sec. 3.2).
     """
 
     def __init__(self, in_features: int, out_features: int, k: int,
-                 bases: Sequence[Tuple[int, int]], device=None, dtype=None):
+                 bases: Sequence[Tuple[int, int]], device=None, dtype=None, bias: bool = False,
+                 save_projected: bool = False):
         super().__init__()
         w = torch.empty((out_features, in_features), device=device, dtype=dtype)
         torch.nn.init.normal_(w, std=in_features ** -0.5)
         self.weight = torch.nn.Parameter(w)
+        self.bias = (torch.nn.Parameter(torch.zeros(out_features, device=device, dtype=dtype))
+                     if bias else None)
         self.k, self.bases = int(k), [tuple(p) for p in bases]
+        self.save_projected = bool(save_projected)
 
     def forward(self, x: torch.Tensor) -> torch.Tensor:
-        return LbpLinearFunction.apply(x, self.weight, self.k, self.bases)
+        return LbpLinearFunction.apply(x, self.weight, self.bias, self.k, self.bases,
+                                       self.save_projected)

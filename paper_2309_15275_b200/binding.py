@@ -41,6 +41,11 @@ class Layer(C.Structure):
                 ("dtype", C.c_int32), ("gw_dtype", C.c_int32)]
 
 
+class Extras(C.Structure):
+    _fields_ = [("beta", C.c_float), ("g_bias", C.c_void_p), ("n_extra", C.c_int32),
+                ("x_extra", C.c_void_p), ("gy_extra", C.c_void_p), ("gx_extra", C.c_void_p)]
+
+
 _LIB = None
 
 
@@ -80,6 +85,14 @@ def _lib() -> C.CDLL:
         lib.lbp_backward.argtypes = [vp, vp, vp, vp, vp, C.POINTER(Layer), C.POINTER(Basis), i32,
                                      vp, sz, vp]
         lib.lbp_backward.restype = i32
+        lib.lbp_workspace_bytes_ex.argtypes = [C.POINTER(Layer), i32, C.POINTER(Extras)]
+        lib.lbp_workspace_bytes_ex.restype = sz
+        lib.lbp_backward_ex.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Layer), C.POINTER(Basis),
+                                        i32, C.POINTER(Extras), vp, sz, vp]
+        lib.lbp_backward_ex.restype = i32
+        lib.lbp_backward_projected.argtypes = [vp, vp, vp, vp, vp, C.POINTER(Layer),
+                                               C.POINTER(Basis), i32, vp, sz, vp]
+        lib.lbp_backward_projected.restype = i32
         lib.lbp_backward_batch.argtypes = [i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
                                            C.POINTER(vp), C.POINTER(vp), C.POINTER(Layer),
                                            C.POINTER(Basis), i32, C.POINTER(vp), C.POINTER(sz),
@@ -92,6 +105,9 @@ def _lib() -> C.CDLL:
         lib.lbp_backward_static.argtypes = [vp, vp, vp, vp, vp, C.POINTER(Layer), C.POINTER(Basis),
                                             i32, vp]
         lib.lbp_backward_static.restype = i32
+        lib.lbp_test_tile_plan.argtypes = [i32] * 9 + [C.POINTER(C.c_int32), C.POINTER(C.c_uint16),
+                                                       C.POINTER(C.c_uint16)]
+        lib.lbp_test_tile_plan.restype = i32
         lib.lbp_test_reload_env.argtypes = []
         lib.lbp_test_reload_env.restype = i32
         lib.lbp_test_stall_products.argtypes = [i32]
@@ -114,7 +130,8 @@ EXPORTED = ("lbp_select_bases", "lbp_basis_matrix", "lbp_flops", "lbp_status_str
             "lbp_backward_static", "lbp_launch_count", "lbp_set_phase_events", "lbp_phase_count",
             "lbp_phase_name", "lbp_select_lhe", "lbp_spectrum_workspace_bytes", "lbp_spectrum",
             "lbp_backward_batch", "lbp_test_stall_products",
-            "lbp_test_reload_env")
+            "lbp_test_reload_env", "lbp_workspace_bytes_ex", "lbp_backward_ex",
+            "lbp_backward_projected", "lbp_test_tile_plan")
 
 
 def _check(status: int, where: str) -> None:
@@ -193,11 +210,12 @@ def _status_ws(device) -> torch.Tensor:
 
 def lbp_project(t: torch.Tensor, k: int, bases, out: torch.Tensor | None = None,
                 ws: torch.Tensor | None = None) -> torch.Tensor:
-    """t (B,H,W,C) -> t_hat (B,H/k,W/k,r,C)."""
+    """t (B,H,W,C) -> t_hat (B,ceil(H/k),ceil(W/k),r,C)."""
     B, H, W, Cc = t.shape
     r = len(bases)
     if out is None:
-        out = torch.empty((B, H // max(k, 1), W // max(k, 1), r, Cc), dtype=t.dtype, device=t.device)
+        kk = max(k, 1)
+        out = torch.empty((B, -(-H // kk), -(-W // kk), r, Cc), dtype=t.dtype, device=t.device)
     if ws is None:
         ws = _status_ws(t.device)
     _check(_lib().lbp_project(_dev(t, "t"), _dev(out, "t_hat"), B, H, W, Cc, k, _bases(bases), r,
@@ -239,14 +257,18 @@ def lbp_spectrum(t: torch.Tensor, k: int, out: torch.Tensor | None = None,
 
 
 def lbp_expand(t_hat: torch.Tensor, k: int, bases, out: torch.Tensor | None = None,
-               ws: torch.Tensor | None = None) -> torch.Tensor:
-    """t_hat (B,H/k,W/k,r,C) -> t (B,H,W,C)."""
+               ws: torch.Tensor | None = None, grid: Tuple[int, int] | None = None) -> torch.Tensor:
+    """t_hat (B,ceil(H/k),ceil(W/k),r,C) -> t (B,H,W,C).  grid = (H, W) when the
+    grid sides are not multiples of k (default: Hb * k, Wb * k)."""
     B, Hb, Wb, r, Cc = t_hat.shape
+    H, W = grid if grid is not None else (Hb * k, Wb * k)
+    if -(-H // max(k, 1)) != Hb or -(-W // max(k, 1)) != Wb:
+        raise ValueError("grid does not match the block grid of t_hat")
     if out is None:
-        out = torch.empty((B, Hb * k, Wb * k, Cc), dtype=t_hat.dtype, device=t_hat.device)
+        out = torch.empty((B, H, W, Cc), dtype=t_hat.dtype, device=t_hat.device)
     if ws is None:
         ws = _status_ws(t_hat.device)
-    _check(_lib().lbp_expand(_dev(t_hat, "t_hat"), _dev(out, "t"), B, Hb * k, Wb * k, Cc, k,
+    _check(_lib().lbp_expand(_dev(t_hat, "t_hat"), _dev(out, "t"), B, H, W, Cc, k,
                              _bases(bases), len(bases), _dtype_code(t_hat.dtype),
                              _dev(ws, "ws"), ws.numel(), _stream()),
            "lbp_expand")
@@ -263,12 +285,44 @@ def alloc_workspace(x: torch.Tensor, g_y: torch.Tensor, k: int, r: int,
     return torch.empty(n, dtype=torch.uint8, device=x.device)
 
 
+def _check_layer_tensors(g_y, W, g_x, g_W, Cin: int, x=None, x_hat=None, k=None, r=None):
+    """Shapes, dtypes and devices of one backward problem, before the C call: the
+    library sees raw pointers and would read a short or mistyped buffer as it is."""
+    if g_y.dim() != 4:
+        raise ValueError("g_y must be (B, H, W, Cout)")
+    B, H, Wd, Cout = g_y.shape
+    dt, dev = g_y.dtype, g_y.device
+    if x is not None and tuple(x.shape) != (B, H, Wd, Cin):
+        raise ValueError(f"x {tuple(x.shape)} does not match g_y {tuple(g_y.shape)} and Cin {Cin}")
+    if x_hat is not None:
+        want = (B, -(-H // max(k, 1)), -(-Wd // max(k, 1)), r, Cin)
+        if tuple(x_hat.shape) != want:
+            raise ValueError(f"x_hat {tuple(x_hat.shape)} must be {want}")
+    if tuple(W.shape) != (Cout, Cin):
+        raise ValueError(f"W {tuple(W.shape)} must be (Cout, Cin) = ({Cout}, {Cin})")
+    if g_x is not None and tuple(g_x.shape) != (B, H, Wd, Cin):
+        raise ValueError(f"g_x {tuple(g_x.shape)} must be {(B, H, Wd, Cin)}")
+    if g_W is not None and tuple(g_W.shape) != (Cout, Cin):
+        raise ValueError(f"g_W {tuple(g_W.shape)} must be ({Cout}, {Cin})")
+    for name, t in (("x", x), ("x_hat", x_hat), ("W", W), ("g_x", g_x)):
+        if t is not None and t.dtype != dt:
+            raise ValueError(f"{name} is {t.dtype}, g_y is {dt}: one dtype per layer")
+    for name, t in (("x", x), ("x_hat", x_hat), ("W", W), ("g_x", g_x), ("g_W", g_W)):
+        if t is not None and t.device != dev:
+            raise ValueError(f"{name} is on {t.device}, g_y on {dev}")
+    if dev.type == "cuda" and dev.index is not None and dev.index != torch.cuda.current_device():
+        raise ValueError(f"tensors are on {dev}, the current device is cuda:{torch.cuda.current_device()}")
+
+
 def lbp_backward(x, g_y, W, k: int, bases, *, gw_dtype: torch.dtype = torch.float32,
                  g_x=None, g_W=None, ws=None):
     """Algorithm 1.  Returns (g_x (B,H,W,Cin), g_W (Cout,Cin))."""
+    if x.dim() != 4:
+        raise ValueError("x must be (B, H, W, Cin)")
     B, H, Wd, Cin = x.shape
     Cout = g_y.shape[-1]
     r = len(bases)
+    _check_layer_tensors(g_y, W, g_x, g_W, Cin, x=x)
     if g_x is None:
         g_x = torch.empty_like(x)
     if g_W is None:
@@ -283,6 +337,103 @@ def lbp_backward(x, g_y, W, k: int, bases, *, gw_dtype: torch.dtype = torch.floa
     return g_x, g_W
 
 
+def _extras(g_y, Cin, beta, g_bias, x_extra, gy_extra, gx_extra):
+    Cout = g_y.shape[-1]
+    ex = Extras()
+    ex.beta = float(beta)
+    if g_bias is not None:
+        if g_bias.dtype != torch.float32 or tuple(g_bias.shape) != (Cout,):
+            raise ValueError("g_bias must be fp32 of shape (Cout,)")
+        ex.g_bias = _dev(g_bias, "g_bias")
+    n = 0
+    if x_extra is not None or gy_extra is not None:
+        if x_extra is None or gy_extra is None or gx_extra is None:
+            raise ValueError("x_extra, gy_extra and gx_extra go together")
+        n = x_extra.shape[0]
+        if (tuple(x_extra.shape) != (n, Cin) or tuple(gy_extra.shape) != (n, Cout)
+                or tuple(gx_extra.shape) != (n, Cin)):
+            raise ValueError("extra tokens must be (n, Cin), (n, Cout), (n, Cin)")
+        for t in (x_extra, gy_extra, gx_extra):
+            if t.dtype != g_y.dtype or t.device != g_y.device:
+                raise ValueError("extra tokens must have the layer's dtype and device")
+        if n > 0:
+            ex.x_extra, ex.gy_extra, ex.gx_extra = (_dev(x_extra, "x_extra"), _dev(gy_extra, "gy_extra"),
+                                                    _dev(gx_extra, "gx_extra"))
+    ex.n_extra = n
+    return ex
+
+
+def lbp_workspace_bytes_ex(B, H, W, Cin, Cout, k, dtype: int, gw_dtype: int, r: int, *, beta=0.0,
+                           bias=False, n_extra=0) -> int:
+    lay = _layer(B, H, W, Cin, Cout, k, dtype, gw_dtype)
+    ex = Extras()
+    ex.beta, ex.n_extra = float(beta), 0
+    # sizes only: the pointers are not looked at beyond NULL / non-NULL
+    ex.g_bias = 16 if bias else None
+    if n_extra:
+        ex.n_extra, ex.x_extra, ex.gy_extra, ex.gx_extra = int(n_extra), 16, 16, 16
+    return int(_lib().lbp_workspace_bytes_ex(C.byref(lay), r, C.byref(ex)))
+
+
+def lbp_backward_ex(x, g_y, W, k: int, bases, *, x_hat=None, beta: float = 0.0, g_bias=None,
+                    x_extra=None, gy_extra=None, gx_extra=None,
+                    gw_dtype: torch.dtype = torch.float32, g_x=None, g_W=None, ws=None):
+    """Algorithm 1 with what a ViT layer needs around it: accumulation into g_W
+    (beta), the bias gradient, tokens outside the grid (Eq. 2), and x_hat = p(x)
+    handed in instead of x (pass x=None).  Returns (g_x, g_W)."""
+    if (x is None) == (x_hat is None):
+        raise ValueError("give exactly one of x and x_hat")
+    B, H, Wd, Cout = g_y.shape
+    r = len(bases)
+    Cin = (x if x is not None else x_hat).shape[-1]
+    _check_layer_tensors(g_y, W, g_x, g_W, Cin, x=x, x_hat=x_hat, k=k, r=r)
+    if g_x is None:
+        g_x = torch.empty((B, H, Wd, Cin), dtype=g_y.dtype, device=g_y.device)
+    if g_W is None:
+        if beta != 0.0:
+            raise ValueError("beta != 0 accumulates into g_W: pass it")
+        g_W = torch.empty((Cout, Cin), dtype=gw_dtype, device=g_y.device)
+    ex = _extras(g_y, Cin, beta, g_bias, x_extra, gy_extra, gx_extra)
+    lay = _layer(B, H, Wd, Cin, Cout, k, _dtype_code(g_y.dtype), _dtype_code(g_W.dtype))
+    if ws is None:
+        n = int(_lib().lbp_workspace_bytes_ex(C.byref(lay), r, C.byref(ex)))
+        if n == 0:
+            raise ValueError("invalid layer for lbp_workspace_bytes_ex")
+        ws = torch.empty(n, dtype=torch.uint8, device=g_y.device)
+    _check(_lib().lbp_backward_ex(None if x is None else _dev(x, "x"),
+                                  None if x_hat is None else _dev(x_hat, "x_hat"),
+                                  _dev(g_y, "g_y"), _dev(W, "W"), _dev(g_x, "g_x"), _dev(g_W, "g_W"),
+                                  C.byref(lay), _bases(bases), r, C.byref(ex), _dev(ws, "ws"),
+                                  ws.numel(), _stream()),
+           "lbp_backward_ex")
+    return g_x, g_W
+
+
+def lbp_backward_projected(x_hat, g_y, W, k: int, bases, *, gw_dtype: torch.dtype = torch.float32,
+                           g_x=None, g_W=None, ws=None):
+    """Algorithm 1 from its second step on: x_hat = lbp_project(x, k, bases) was
+    taken at forward time (Eq. 3).  Returns (g_x, g_W)."""
+    B, H, Wd, Cout = g_y.shape
+    r = len(bases)
+    Cin = x_hat.shape[-1]
+    _check_layer_tensors(g_y, W, g_x, g_W, Cin, x_hat=x_hat, k=k, r=r)
+    if g_x is None:
+        g_x = torch.empty((B, H, Wd, Cin), dtype=g_y.dtype, device=g_y.device)
+    if g_W is None:
+        g_W = torch.empty((Cout, Cin), dtype=gw_dtype, device=g_y.device)
+    lay = _layer(B, H, Wd, Cin, Cout, k, _dtype_code(g_y.dtype), _dtype_code(g_W.dtype))
+    if ws is None:
+        n = int(_lib().lbp_workspace_bytes(C.byref(lay), r))
+        if n == 0:
+            raise ValueError("invalid layer for lbp_workspace_bytes")
+        ws = torch.empty(n, dtype=torch.uint8, device=g_y.device)
+    _check(_lib().lbp_backward_projected(_dev(x_hat, "x_hat"), _dev(g_y, "g_y"), _dev(W, "W"),
+                                         _dev(g_x, "g_x"), _dev(g_W, "g_W"), C.byref(lay),
+                                         _bases(bases), r, _dev(ws, "ws"), ws.numel(), _stream()),
+           "lbp_backward_projected", "lbp_test_tile_plan")
+    return g_x, g_W
+
+
 def lbp_backward_batch(xs, g_ys, Ws, k: int, bases, *, g_xs, g_Ws, wss, done_events=None):
     """Algorithm 1 for several independent layers in one call (same k and bases).
     Every argument is a list with one tensor per layer; outputs and workspaces are
@@ -292,6 +443,7 @@ def lbp_backward_batch(xs, g_ys, Ws, k: int, bases, *, g_xs, g_Ws, wss, done_eve
     n = len(xs)
     lays = (Layer * n)()
     for i in range(n):
+        _check_layer_tensors(g_ys[i], Ws[i], g_xs[i], g_Ws[i], xs[i].shape[-1], x=xs[i])
         B, H, Wd, Cin = xs[i].shape
         lays[i] = _layer(B, H, Wd, Cin, g_ys[i].shape[-1], k, _dtype_code(xs[i].dtype),
                          _dtype_code(g_Ws[i].dtype))
@@ -319,6 +471,7 @@ def lbp_backward_fullrank(x, g_y, W, k: int, *, gw_dtype: torch.dtype = torch.fl
     """Eq. 2, exact backpropagation (the r = k*k mode)."""
     B, H, Wd, Cin = x.shape
     Cout = g_y.shape[-1]
+    _check_layer_tensors(g_y, W, g_x, g_W, Cin, x=x)
     if g_x is None:
         g_x = torch.empty_like(x)
     if g_W is None:
@@ -343,6 +496,7 @@ def lbp_backward_static(x, g_y, W, k: int, bases, *, g_x, g_W):
     STATIC_SCRATCH_BYTES raise LbpError (status 7)."""
     B, H, Wd, Cin = x.shape
     Cout = g_y.shape[-1]
+    _check_layer_tensors(g_y, W, g_x, g_W, Cin, x=x)
     lay = _layer(B, H, Wd, Cin, Cout, k, _dtype_code(x.dtype), _dtype_code(g_W.dtype))
     _check(_lib().lbp_backward_static(_dev(x, "x"), _dev(g_y, "g_y"), _dev(W, "W"),
                                       _dev(g_x, "g_x"), _dev(g_W, "g_W"), C.byref(lay),
@@ -356,6 +510,20 @@ def lbp_poll_status(ws: torch.Tensor) -> int:
     return int(_lib().lbp_poll_status(_dev(ws, "ws"), _stream()))
 
 
+def lbp_test_tile_plan(Cin, Cout, G, bpt, k, units, pair, max_splits=1, epi_kind=0):
+    """Test hook: the host-side tile plan of the products kernel.  Returns
+    (dict of tile sizes, list of per-unit tile-id lists or None when not listed)."""
+    out = (C.c_int32 * 6)()
+    first = (C.c_uint16 * 161)()
+    ids = (C.c_uint16 * 1536)()
+    _check(_lib().lbp_test_tile_plan(Cin, Cout, G, bpt, k, units, 1 if pair else 0, max_splits,
+                                     epi_kind, out, first, ids), "lbp_test_tile_plan")
+    info = {"BNw": out[0], "BNx": out[1], "splits": out[2], "kbps": out[3], "listed": bool(out[4])}
+    if not info["listed"]:
+        return info, None
+    return info, [[ids[j] for j in range(first[u], first[u + 1])] for u in range(units)]
+
+
 def lbp_test_reload_env() -> None:
     """Test hook: the library reads its LBP_* tuning switches from the environment again."""
     _check(_lib().lbp_test_reload_env(), "lbp_test_reload_env")
@@ -364,8 +532,7 @@ def lbp_test_reload_env() -> None:
 def lbp_test_stall_products(on: bool) -> None:
     """Test hook (include/lbp_test_hooks.h): while on, the products kernel's TMA
     producers issue nothing, so the call ends in LBP_ERR_TIMEOUT (lbp_poll_status)."""
-    _check(_lib().lbp_test_stall_products(1 if on else 0), "lbp_test_stall_products",
-            "lbp_test_reload_env")
+    _check(_lib().lbp_test_stall_products(1 if on else 0), "lbp_test_stall_products")
 
 
 # ------------------------------------------------------ measurement hooks ----

@@ -3,7 +3,11 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
+#include <cstdio>
 #include <cstdlib>
+#include <cstring>
+#include <mutex>
 
 #include "lbp_fused.cuh"
 #include "lbp_internal.h"
@@ -114,7 +118,6 @@ static int check_grid(int B, int H, int W, int C, int k, int dtype) {
   if (int e = check_order(k)) return e;
   if (dtype != LBP_F32 && dtype != LBP_BF16) return LBP_ERR_DTYPE;
   if (B <= 0 || H <= 0 || W <= 0 || C <= 0) return LBP_ERR_SHAPE;
-  if (H % k != 0 || W % k != 0) return LBP_ERR_SHAPE;
   if ((static_cast<long long>(C) * elem_size(dtype)) % 16 != 0) return LBP_ERR_ALIGN;
   return LBP_OK;
 }
@@ -134,6 +137,31 @@ struct Layout {
   long long rows;   // M_hat = blocks * r
 };
 
+// Scratch of lbp_backward_ex beyond `Layout::total`: two fp32 (Cout, Cin)
+// matrices (this call's g_W before it is added to the caller's, the term of the
+// tokens outside the grid) and the fp64 column-sum partials of the bias gradient.
+struct ExtrasLayout {
+  size_t gw0, gw1, bias_a, bias_b, total;
+};
+constexpr int kBiasSlabsMax = 64;
+
+static ExtrasLayout plan_extras(const lbp_layer& L, size_t base_total) {
+  ExtrasLayout e{};
+  size_t off = align_up(base_total, 1024);
+  const size_t gw = static_cast<size_t>(L.Cout) * L.Cin * 4;
+  e.gw0 = off;
+  off = align_up(off + gw, 1024);
+  e.gw1 = off;
+  off = align_up(off + gw, 1024);
+  const size_t part = static_cast<size_t>(kBiasSlabsMax) * L.Cout * 8;
+  e.bias_a = off;
+  off = align_up(off + part, 1024);
+  e.bias_b = off;
+  off = align_up(off + part, 1024);
+  e.total = off;
+  return e;
+}
+
 // The persistent products kernel can be switched off (LBP_FUSED=0) to run the
 // separate product and expansion kernels instead.
 static bool fused_enabled() { return tune_options().fused; }
@@ -141,7 +169,8 @@ static bool fused_enabled() { return tune_options().fused; }
 static Layout plan_layout(const lbp_layer& L, int r) {
   Layout w{};
   const long long T = static_cast<long long>(L.B) * L.H * L.W;
-  const long long nb = T / (L.k * L.k);
+  // blocks of the grid extended with zero tokens to multiples of k
+  const long long nb = static_cast<long long>(L.B) * blocks_along(L.H, L.k) * blocks_along(L.W, L.k);
   const int es = elem_size(L.dtype);
   size_t off = kStatusBytes;
   if (r < L.k * L.k) {
@@ -230,7 +259,8 @@ int lbp_project(const void* t, void* t_hat, int B, int H, int W, int C, int k,
 size_t lbp_spectrum_workspace_bytes(int B, int H, int W, int C, int k, int dtype) {
   if (check_grid(B, H, W, C, k, dtype) != LBP_OK) return 0;
   const size_t es = dtype == LBP_BF16 ? 2 : 4;
-  const size_t coef = static_cast<size_t>(B) * H * W * C * es;   // all k*k coefficients per block
+  // all k*k coefficients per block of the zero-extended grid
+  const size_t coef = static_cast<size_t>(B) * blocks_along(H, k) * blocks_along(W, k) * k * k * C * es;
   return kStatusBytes + (coef + 255) / 256 * 256;
 }
 
@@ -257,7 +287,7 @@ int lbp_spectrum(const void* t, double* energy, int B, int H, int W, int C, int 
   if (int e = launch_project(t, coef, dtype, B, H, W, C, plan, RowMap{1, r},
                              static_cast<uint32_t*>(ws), st))
     return e;
-  const long long rows = static_cast<long long>(B) * H * W;   // blocks * k * k
+  const long long rows = static_cast<long long>(B) * blocks_along(H, k) * blocks_along(W, k) * k * k;
   return launch_square_reduce(coef, dtype, rows, C, r, energy, st);
 }
 
@@ -293,6 +323,169 @@ static int validate_backward(const void* x, const void* g_y, const void* W, cons
 }  // extern "C"
 
 namespace lbp {
+
+// Stream and events of the library's own for lbp_backward_batch, one set per
+// device, created at the first batch call on that device and kept.
+struct SideStream {
+  cudaStream_t stream;
+  cudaEvent_t fork;
+  cudaEvent_t done[64];
+};
+static int side_stream(SideStream** out) {
+  static SideStream per_device[64];
+  static bool ready[64] = {};
+  static std::mutex mu;
+  int dev = 0;
+  LBP_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return LBP_ERR_ARCH;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!ready[dev]) {
+    SideStream& s = per_device[dev];
+    LBP_CUDA_TRY(cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking));
+    LBP_CUDA_TRY(cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming));
+    for (int i = 0; i < 64; ++i)
+      LBP_CUDA_TRY(cudaEventCreateWithFlags(&s.done[i], cudaEventDisableTiming));
+    ready[dev] = true;
+  }
+  *out = &per_device[dev];
+  return LBP_OK;
+}
+
+// How lbp_backward_batch runs its problems: in which order, whether the
+// projections go to the side stream, and how many SMs the projection at each
+// position gets beside the products kernel before it.
+struct BatchPlan {
+  bool side;
+  int sms;
+  int order[64];
+  int proj_sms[64];   // by position; 0 = all SMs
+};
+
+static int plan_batch(int n, const lbp_layer* layers, const lbp_basis* set, int r, BatchPlan* out) {
+  BatchPlan& bp = *out;
+  bp.side = false;
+  bp.sms = 0;
+  for (int i = 0; i < n; ++i) {
+    bp.order[i] = i;
+    bp.proj_sms[i] = 0;
+  }
+  const int want = tune_options().batch_proj_sms;
+  if (n < 2 || !fused_enabled() || want == 0 || r > 16) return LBP_OK;
+  if (int e = check_device_arch()) return e;
+  int dev = 0, sms = 0;
+  LBP_CUDA_TRY(cudaGetDevice(&dev));
+  LBP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  if (sms < 96) return LBP_OK;
+  bp.sms = sms;
+
+  // recent answers (the search below evaluates the cost models many times)
+  struct Key {
+    int n, r, sms, want;
+    lbp_layer layers[8];
+    lbp_basis set[16];
+    BatchPlan plan;
+  };
+  static thread_local Key cache[8];
+  static thread_local int cache_n = 0, cache_next = 0;
+  const bool keyed = n <= 8;
+  auto same = [&](const Key& k) {
+    if (k.n != n || k.r != r || k.sms != sms || k.want != want) return false;
+    for (int i = 0; i < n; ++i)
+      if (std::memcmp(&k.layers[i], &layers[i], sizeof(lbp_layer)) != 0) return false;
+    for (int q = 0; q < r; ++q)
+      if (k.set[q].i != set[q].i || k.set[q].j != set[q].j) return false;
+    return true;
+  };
+  if (keyed)
+    for (int c = 0; c < cache_n; ++c)
+      if (same(cache[c])) {
+        bp = cache[c].plan;
+        return LBP_OK;
+      }
+
+  BasisPlan plans[64];
+  for (int i = 0; i < n; ++i) {
+    if (make_basis_plan(layers[i].k, set, r, &plans[i]) != LBP_OK || r >= layers[i].k * layers[i].k ||
+        !fused_supported(layers[i], plans[i]) || !fused_pair_supported(layers[i], sms))
+      return LBP_OK;   // a problem that takes another path: one stream, given order
+  }
+  bp.side = true;
+
+  // cost of running problem a's products kernel beside problem b's projection,
+  // and the SM split that gives it
+  auto pair_cost = [&](int a, int b, int* ps_out) {
+    double best = -1.0;
+    int lo = 40, hi = sms - 40;
+    if (want > 0) lo = hi = want & ~1;
+    for (int ps = lo; ps <= hi; ps += 4) {
+      const double tp = fused_projection_model_us(layers[b], plans[b], ps);
+      const double tq = fused_products_model_us(layers[a], plans[a], (sms - ps) / 2);
+      const double t = tp > tq ? tp : tq;
+      if (best < 0 || t < best) {
+        best = t;
+        *ps_out = ps;
+      }
+    }
+    return best;
+  };
+  if (n <= 6) {
+    // every order: first projection alone + pairs + last products kernel alone
+    static thread_local double pc[6][6];
+    static thread_local int pps[6][6];
+    double first[6], last[6];
+    for (int a = 0; a < n; ++a) {
+      first[a] = fused_projection_model_us(layers[a], plans[a], sms);
+      last[a] = fused_products_model_us(layers[a], plans[a], sms / 2);
+      for (int b = 0; b < n; ++b)
+        if (a != b) pc[a][b] = pair_cost(a, b, &pps[a][b]);
+    }
+    int perm[6], best_perm[6];
+    for (int i = 0; i < n; ++i) perm[i] = best_perm[i] = i;
+    double best = -1.0;
+    do {
+      double t = first[perm[0]] + last[perm[n - 1]];
+      for (int i = 0; i + 1 < n; ++i) t += pc[perm[i]][perm[i + 1]];
+      if (best < 0 || t < best - 1e-9) {
+        best = t;
+        for (int i = 0; i < n; ++i) best_perm[i] = perm[i];
+      }
+    } while (std::next_permutation(perm, perm + n));
+    if (tune_options().verbose) {
+      for (int a = 0; a < n; ++a) {
+        fprintf(stderr, "lbp batch model: problem %d projection alone %.1f, products alone %.1f; beside:", a,
+                first[a], last[a]);
+        for (int b = 0; b < n; ++b)
+          if (a != b) fprintf(stderr, " [%d] %.1f @%d", b, pc[a][b], pps[a][b]);
+        fprintf(stderr, "\n");
+      }
+    }
+    for (int i = 0; i < n; ++i) bp.order[i] = best_perm[i];
+    for (int i = 1; i < n; ++i) bp.proj_sms[i] = pps[best_perm[i - 1]][best_perm[i]];
+  } else {
+    for (int i = 1; i < n; ++i) pair_cost(i - 1, i, &bp.proj_sms[i]);
+  }
+  if (tune_options().verbose) {
+    fprintf(stderr, "lbp batch: order");
+    for (int i = 0; i < n; ++i) fprintf(stderr, " %d", bp.order[i]);
+    fprintf(stderr, "; SMs of each projection beside the products kernel before it:");
+    for (int i = 1; i < n; ++i) fprintf(stderr, " %d", bp.proj_sms[i]);
+    fprintf(stderr, "\n");
+  }
+  if (keyed) {
+    Key& k = cache[cache_next];
+    k.n = n;
+    k.r = r;
+    k.sms = sms;
+    k.want = want;
+    for (int i = 0; i < n; ++i) k.layers[i] = layers[i];
+    for (int q = 0; q < r; ++q) k.set[q] = set[q];
+    k.plan = bp;
+    cache_next = (cache_next + 1) % 8;
+    if (cache_n < 8) ++cache_n;
+  }
+  return LBP_OK;
+}
+
 int validate_backward_call(const void* x, const void* g_y, const void* W, const void* g_x,
                            const void* g_W, const lbp_layer* layer, const lbp_basis* set, int r,
                            const void* ws, size_t ws_bytes) {
@@ -303,6 +496,36 @@ int validate_backward_call(const void* x, const void* g_y, const void* W, const 
 }  // namespace lbp
 
 extern "C" {
+
+int lbp_test_tile_plan(int Cin, int Cout, int G, int bpt, int k, int units, int pair,
+                       int max_splits, int epi_kind, int32_t* out6, uint16_t* first, uint16_t* ids) {
+  if (out6 == nullptr || first == nullptr || ids == nullptr) return LBP_ERR_NULL;
+  if (Cin < 1 || Cout < 1 || G < 1 || bpt < 1 || units < 1 || units > kSchedMaxUnits ||
+      epi_kind < 0 || epi_kind > 2)
+    return LBP_ERR_SHAPE;
+  PlanShape s{};
+  s.Cin = Cin;
+  s.Cout = Cout;
+  s.G = G;
+  s.bpt = bpt;
+  s.k = k;
+  s.units = units;
+  s.pair = pair ? 1 : 0;
+  s.max_splits = max_splits;
+  s.epi_kind = epi_kind;
+  s.num_kb_w = G * 2;
+  s.num_kb_x = (Cout + 63) / 64;
+  const TilePlan& t = plan_products(s);
+  out6[0] = t.BNw;
+  out6[1] = t.BNx;
+  out6[2] = t.splits;
+  out6[3] = t.kbps;
+  out6[4] = t.sched.listed;
+  out6[5] = t.sched.listed ? t.sched.first[kSchedMaxUnits] : 0;
+  for (int i = 0; i <= kSchedMaxUnits; ++i) first[i] = t.sched.first[i];
+  for (int i = 0; i < kSchedMaxItems; ++i) ids[i] = t.sched.ids[i];
+  return LBP_OK;
+}
 
 int lbp_test_reload_env(void) {
   reload_tune_options();
@@ -355,14 +578,46 @@ int lbp_backward_batch(int n, const void* const* x, const void* const* g_y, cons
           if (overlap(out[i][a], in[j][b]) || (i < j && overlap(out[i][a], out[j][b])))
             return LBP_ERR_OVERLAP;
     }
+  // Side-stream mode.  The projection streams x and g_y from HBM, the products
+  // kernel lives on operands that sit in L2: run beside each other on disjoint
+  // SMs they use different parts of the machine.  The projections of all problems
+  // go to a stream of the library's own, one after the other; the projection of
+  // the next problem gets some of the SMs while the products kernel of a problem
+  // runs on the others (on the caller's stream, behind an event of its
+  // projection).  The problems are independent, so they are taken in the order
+  // that hides most: what stays exposed is the first projection and the last
+  // products kernel.
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  BatchPlan bplan;
+  if (int e = plan_batch(n, layers, set, r, &bplan)) return e;
+  const bool side = bplan.side;
+  SideStream* ss = nullptr;
+  if (side) {
+    if (int e = side_stream(&ss)) return e;
+    // everything enqueued so far on the caller's stream comes before the first projection
+    LBP_CUDA_TRY(cudaEventRecord(ss->fork, st));
+    LBP_CUDA_TRY(cudaStreamWaitEvent(ss->stream, ss->fork, 0));
+  }
   int status = LBP_OK;
-  for (int i = 0; i < n && status == LBP_OK; ++i) {
-    // From the second problem on, the projection kernel need not wait for the
-    // kernel ahead of it (the previous problem's products kernel): it starts on
-    // the SMs that kernel has already left.
-    set_projection_defer_wait(i > 0);
+  for (int pos = 0; pos < n && status == LBP_OK; ++pos) {
+    const int i = bplan.order[pos];
+    FusedOverlap ov{};
+    if (side) {
+      ov.proj_stream = ss->stream;
+      ov.proj_done = ss->done[pos];
+      ov.proj_ctas = bplan.proj_sms[pos];   // 0 (all SMs) for the first one: nothing runs beside it
+      // nor beside the last products kernel
+      ov.prod_units = pos == n - 1 ? 0 : (bplan.sms - bplan.proj_sms[pos + 1]) / 2;
+      set_fused_overlap(&ov);
+    } else {
+      // One stream: from the second problem on, the projection kernel need not wait
+      // for the kernel ahead of it (the previous problem's products kernel): it
+      // starts on the SMs that kernel has already left.
+      set_projection_defer_wait(pos > 0);
+    }
     status = lbp_backward(x[i], g_y[i], W[i], g_x[i], g_W[i], &layers[i], set, r, ws[i],
                           ws_bytes[i], stream);
+    set_fused_overlap(nullptr);
     if (status == LBP_OK && done_events != nullptr && done_events[i] != nullptr) {
       const cudaError_t ce = cudaEventRecord(static_cast<cudaEvent_t>(done_events[i]),
                                              static_cast<cudaStream_t>(stream));
@@ -376,21 +631,34 @@ int lbp_backward_batch(int n, const void* const* x, const void* const* g_y, cons
   return status;
 }
 
-int lbp_backward(const void* x, const void* g_y, const void* W, void* g_x, void* g_W,
-                 const lbp_layer* layer, const lbp_basis* set, int r, void* ws, size_t ws_bytes,
-                 void* stream) {
-  BasisPlan plan;
-  Layout lay;
-  if (int e = validate_backward(x, g_y, W, g_x, g_W, layer, set, r, ws, ws_bytes, &plan, &lay))
-    return e;
-  const lbp_layer& L = *layer;
-  if (int e = check_device_arch()) return e;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  uint8_t* wsb = static_cast<uint8_t*>(ws);
-  if (r == L.k * L.k) return run_fullrank(x, g_y, W, g_x, g_W, L, wsb, st);
+}  // extern "C"
+
+namespace lbp {
+
+// Where g_y_hat of a call lies (for the bias gradient): null when the call ran
+// the full-rank mode and materialised nothing.
+struct CoefLoc {
+  const void* ptr;
+  RowMap rows;
+  double dc_to_sum;   // token sum of a block = dc_to_sum * its (0,0) coefficient as stored
+};
+
+// Algorithm 1 after validation.  Exactly one of x / x_hat is given: x_hat are the
+// dense coefficients p(x), (blocks * r, Cin), taken earlier (Eq. 3).
+static int run_core(const void* x, const void* x_hat_in, const void* g_y, const void* W, void* g_x,
+                    void* g_W, const lbp_layer& L, const BasisPlan& plan, const Layout& lay,
+                    uint8_t* wsb, cudaStream_t st, CoefLoc* gy_loc) {
+  const int r = plan.r;
+  gy_loc->ptr = nullptr;
+  if (r == L.k * L.k && x_hat_in == nullptr) return run_fullrank(x, g_y, W, g_x, g_W, L, wsb, st);
 
   uint32_t* status = reinterpret_cast<uint32_t*>(wsb);
   if (fused_enabled() && fused_supported(L, plan)) {
+    FusedLayout fl;
+    fused_scratch_bytes(L, r, &fl);
+    gy_loc->ptr = wsb + lay.fused + fl.gy_hat;
+    gy_loc->rows = RowMap{fl.bpt, 128};
+    gy_loc->dc_to_sum = 1.0 / static_cast<double>(fused_scale_gy(L.k));
     // projection kernel, then one persistent kernel for both products with the
     // expansion fused into the g_x_hat epilogue
     if (int e = mark_phase(0, st)) return e;
@@ -398,24 +666,33 @@ int lbp_backward(const void* x, const void* g_y, const void* W, void* g_x, void*
       if (int e = mark_phase(1, s)) return e;
       return mark_phase(2, s);
     };
-    if (int e = launch_fused(x, g_y, W, g_x, g_W, L, plan, wsb + lay.fused, status, st,
+    if (int e = launch_fused(x, x_hat_in, g_y, W, g_x, g_W, L, plan, wsb + lay.fused, status, st,
                              after_projection, nullptr))
       return e;
     for (int ph = 3; ph <= 5; ++ph)
       if (int e = mark_phase(ph, st)) return e;
     return LBP_OK;
   }
-  void* x_hat = wsb + lay.x_hat;
+  const void* x_hat = x_hat_in != nullptr ? x_hat_in : wsb + lay.x_hat;
   void* gy_hat = wsb + lay.gy_hat;
   float* gx_hat = reinterpret_cast<float*>(wsb + lay.gx_hat);
   float* sk = reinterpret_cast<float*>(wsb + lay.splitk);
   const RowMap dense{1, r};
+  gy_loc->ptr = gy_hat;
+  gy_loc->rows = dense;
+  gy_loc->dc_to_sum = static_cast<double>(L.k);   // orthonormal: coefficient = block sum / k
 
   if (int e = mark_phase(0, st)) return e;
-  // Algorithm 1, steps 1-2: x_hat = p(x), g_y_hat = p(g_y), one launch for both
-  if (int e = launch_project2(g_y, gy_hat, L.Cout, x, x_hat, L.Cin, L.dtype, L.B, L.H, L.W, plan,
-                              dense, status, st))
-    return e;
+  if (x_hat_in != nullptr) {
+    // x_hat was taken at forward time: only g_y is projected
+    if (int e = launch_project(g_y, gy_hat, L.dtype, L.B, L.H, L.W, L.Cout, plan, dense, status, st))
+      return e;
+  } else {
+    // Algorithm 1, steps 1-2: x_hat = p(x), g_y_hat = p(g_y), one launch for both
+    if (int e = launch_project2(g_y, gy_hat, L.Cout, x, wsb + lay.x_hat, L.Cin, L.dtype, L.B, L.H,
+                                L.W, plan, dense, status, st))
+      return e;
+  }
   if (int e = mark_phase(1, st)) return e;
   if (int e = mark_phase(2, st)) return e;
   // step 3: g_W = g_y_hat^T x_hat
@@ -433,6 +710,130 @@ int lbp_backward(const void* x, const void* g_y, const void* W, void* g_x, void*
                             dense, st))
     return e;
   return mark_phase(5, st);
+}
+
+static int check_extras(const lbp_extras* ex) {
+  if (ex == nullptr) return LBP_OK;
+  if (!(ex->beta == ex->beta)) return LBP_ERR_SHAPE;   // NaN
+  if (ex->n_extra < 0) return LBP_ERR_SHAPE;
+  if (ex->n_extra > 0) {
+    if (ex->x_extra == nullptr || ex->gy_extra == nullptr || ex->gx_extra == nullptr)
+      return LBP_ERR_NULL;
+    if (!aligned16(ex->x_extra) || !aligned16(ex->gy_extra) || !aligned16(ex->gx_extra))
+      return LBP_ERR_ALIGN;
+  }
+  if (ex->g_bias != nullptr && !aligned16(ex->g_bias)) return LBP_ERR_ALIGN;
+  return LBP_OK;
+}
+
+// lbp_backward_ex after validation.
+static int run_backward_ex(const void* x, const void* x_hat, const void* g_y, const void* W,
+                           void* g_x, void* g_W, const lbp_layer& L, const BasisPlan& plan,
+                           const Layout& lay, const lbp_extras* ex, uint8_t* wsb, cudaStream_t st) {
+  CoefLoc gy_loc{};
+  const bool accumulate = ex != nullptr && (ex->beta != 0.f || ex->n_extra > 0);
+  if (!accumulate && (ex == nullptr || ex->g_bias == nullptr))
+    return run_core(x, x_hat, g_y, W, g_x, g_W, L, plan, lay, wsb, st, &gy_loc);
+
+  const ExtrasLayout el = plan_extras(L, lay.total);
+  uint32_t* status = reinterpret_cast<uint32_t*>(wsb);
+  float* gw0 = reinterpret_cast<float*>(wsb + el.gw0);
+  float* gw1 = reinterpret_cast<float*>(wsb + el.gw1);
+  float* sk = reinterpret_cast<float*>(wsb + lay.splitk);
+  lbp_layer Lg = L;
+  if (accumulate) Lg.gw_dtype = LBP_F32;   // this call's term in fp32, added below
+  if (int e = run_core(x, x_hat, g_y, W, g_x, accumulate ? static_cast<void*>(gw0) : g_W, Lg, plan,
+                       lay, wsb, st, &gy_loc))
+    return e;
+  if (ex->n_extra > 0) {
+    // tokens outside the grid (a class token): Eq. 2 exactly
+    if (int e = launch_gemm(ex->gy_extra, /*a_mn_major=*/true, ex->x_extra, gw1, L.dtype, LBP_F32,
+                            L.Cout, L.Cin, ex->n_extra, sk, lay.splitk_bytes, status, st))
+      return e;
+    if (int e = launch_gemm(ex->gy_extra, /*a_mn_major=*/false, W, ex->gx_extra, L.dtype, L.dtype,
+                            ex->n_extra, L.Cin, L.Cout, sk, lay.splitk_bytes, status, st))
+      return e;
+  }
+  if (accumulate)
+    if (int e = launch_gw_combine(g_W, L.gw_dtype == LBP_BF16, gw0, ex->n_extra > 0 ? gw1 : nullptr,
+                                  ex->beta, static_cast<long long>(L.Cout) * L.Cin, st))
+      return e;
+  if (ex->g_bias != nullptr) {
+    // Sum of g_y over all tokens.  With the DC basis (0,0) selected that is k times
+    // the sum of the DC coefficients of g_y_hat, which the call has just produced;
+    // otherwise g_y is read once more.
+    double* pa = reinterpret_cast<double*>(wsb + el.bias_a);
+    double* pb = reinterpret_cast<double*>(wsb + el.bias_b);
+    int q_dc = -1;
+    for (int q = 0; q < plan.r; ++q)
+      if (plan.seq_i[q] == 0 && plan.seq_j[q] == 0) q_dc = q;
+    long long n_a;
+    double scale_a;
+    if (gy_loc.ptr != nullptr && q_dc >= 0) {
+      n_a = static_cast<long long>(L.B) * blocks_along(L.H, L.k) * blocks_along(L.W, L.k);
+      scale_a = gy_loc.dc_to_sum;
+      if (int e = launch_column_sum(gy_loc.ptr, L.dtype, n_a, L.Cout, gy_loc.rows, plan.r, q_dc, pa, st))
+        return e;
+    } else {
+      n_a = static_cast<long long>(L.B) * L.H * L.W;
+      scale_a = 1.0;
+      if (int e = launch_column_sum(g_y, L.dtype, n_a, L.Cout, RowMap{1, 1}, 0, 0, pa, st)) return e;
+    }
+    if (ex->n_extra > 0)
+      if (int e = launch_column_sum(ex->gy_extra, L.dtype, ex->n_extra, L.Cout, RowMap{1, 1}, 0, 0, pb, st))
+        return e;
+    if (int e = launch_bias_finish(static_cast<float*>(ex->g_bias), L.Cout, ex->beta, pa,
+                                   bias_slabs(n_a), scale_a, pb, bias_slabs(ex->n_extra), st))
+      return e;
+  }
+  return LBP_OK;
+}
+
+}  // namespace lbp
+
+extern "C" {
+
+int lbp_backward(const void* x, const void* g_y, const void* W, void* g_x, void* g_W,
+                 const lbp_layer* layer, const lbp_basis* set, int r, void* ws, size_t ws_bytes,
+                 void* stream) {
+  BasisPlan plan;
+  Layout lay;
+  if (int e = validate_backward(x, g_y, W, g_x, g_W, layer, set, r, ws, ws_bytes, &plan, &lay))
+    return e;
+  if (int e = check_device_arch()) return e;
+  CoefLoc loc{};
+  return run_core(x, nullptr, g_y, W, g_x, g_W, *layer, plan, lay, static_cast<uint8_t*>(ws),
+                  static_cast<cudaStream_t>(stream), &loc);
+}
+
+size_t lbp_workspace_bytes_ex(const lbp_layer* layer, int r, const lbp_extras* ex) {
+  const size_t base = lbp_workspace_bytes(layer, r);
+  if (base == 0 || check_extras(ex) != LBP_OK) return 0;
+  if (ex == nullptr || (ex->beta == 0.f && ex->n_extra == 0 && ex->g_bias == nullptr)) return base;
+  return plan_extras(*layer, base).total;
+}
+
+int lbp_backward_ex(const void* x, const void* x_hat, const void* g_y, const void* W, void* g_x,
+                    void* g_W, const lbp_layer* layer, const lbp_basis* set, int r,
+                    const lbp_extras* ex, void* ws, size_t ws_bytes, void* stream) {
+  if ((x == nullptr) == (x_hat == nullptr)) return LBP_ERR_NULL;   // exactly one of the two
+  const void* xin = x != nullptr ? x : x_hat;
+  BasisPlan plan;
+  Layout lay;
+  if (int e = validate_backward(xin, g_y, W, g_x, g_W, layer, set, r, ws, ws_bytes, &plan, &lay))
+    return e;
+  if (int e = check_extras(ex)) return e;
+  if (ws_bytes < lbp_workspace_bytes_ex(layer, r, ex)) return LBP_ERR_WORKSPACE;
+  if (int e = check_device_arch()) return e;
+  return run_backward_ex(x, x_hat, g_y, W, g_x, g_W, *layer, plan, lay, ex,
+                         static_cast<uint8_t*>(ws), static_cast<cudaStream_t>(stream));
+}
+
+int lbp_backward_projected(const void* x_hat, const void* g_y, const void* W, void* g_x, void* g_W,
+                           const lbp_layer* layer, const lbp_basis* set, int r, void* ws,
+                           size_t ws_bytes, void* stream) {
+  return lbp_backward_ex(nullptr, x_hat, g_y, W, g_x, g_W, layer, set, r, nullptr, ws, ws_bytes,
+                         stream);
 }
 
 int lbp_backward_fullrank(const void* x, const void* g_y, const void* W, void* g_x, void* g_W,

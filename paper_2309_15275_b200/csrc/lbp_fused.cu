@@ -50,7 +50,7 @@ __device__ __forceinline__ void trace_mark(const FusedParams& p, int slot, bool 
   if (p.trace != nullptr) {
     unsigned long long now;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
-    unsigned long long* t = p.trace + blockIdx.x * 8 + slot;
+    unsigned long long* t = p.trace + blockIdx.x * kTraceSlots + slot;
     if (first_only) {
       if (*t == 0) *t = now;
     } else {
@@ -62,62 +62,6 @@ __device__ __forceinline__ void trace_mark(const FusedParams& p, int slot, bool 
 #endif
 }
 
-// Tile list.  Tiles are numbered with the GW tiles (the larger ones) first and
-// dealt to the CTAs in a snake: first pass forwards, second pass backwards, ... so
-// that a CTA that got a large tile gets its next one last.  A CTA takes its
-// tiles in list order (walking the list backwards, GX tiles first, measured no
-// faster).
-struct Tile {
-  int is_gw;
-  int a, b;          // GW: (i, j) ; GX: (m, n)
-  int kb0, n_kb;     // k-block range of the tile (a K slice for GW)
-  int slice;
-};
-__device__ __forceinline__ int tiles_of_cta(const FusedParams& p, int cta, int grid) {
-  const int total = p.n_gw_tiles + p.n_gx_tiles;
-  int n = 0;
-  for (int round = 0; round * grid < total; ++round) {
-    const int pos = (round & 1) ? (grid - 1 - cta) : cta;
-    if (round * grid + pos < total) ++n;
-  }
-  return n;
-}
-__device__ __forceinline__ Tile nth_tile(const FusedParams& p, int cta, int grid, int nth) {
-  const int total = p.n_gw_tiles + p.n_gx_tiles;
-  int seen = 0, id = 0;
-  for (int round = 0; round * grid < total; ++round) {
-    const int pos = (round & 1) ? (grid - 1 - cta) : cta;
-    const int t = round * grid + pos;
-    if (t < total) {
-      if (seen == nth) {
-        id = t;
-        break;
-      }
-      ++seen;
-    }
-  }
-  Tile tl;
-  if (id < p.n_gw_tiles) {
-    tl.is_gw = 1;
-    const int t = id / p.gw_splits;
-    tl.slice = id - t * p.gw_splits;
-    tl.a = t / p.nt_w;
-    tl.b = t - tl.a * p.nt_w;
-    tl.kb0 = tl.slice * p.kb_per_split_w;
-    const int end = tl.kb0 + p.kb_per_split_w;
-    tl.n_kb = (end < p.num_kb_w ? end : p.num_kb_w) - tl.kb0;
-  } else {
-    id -= p.n_gw_tiles;
-    tl.is_gw = 0;
-    tl.slice = 0;
-    tl.a = id / p.n_tx;
-    tl.b = id - tl.a * p.n_tx;
-    tl.kb0 = 0;
-    tl.n_kb = p.num_kb_x;
-  }
-  return tl;
-}
-
 // ------------------------------------------------------------------ kernel ----
 template <int K, int LB, int NEX = 0>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -126,7 +70,8 @@ __global__ void __launch_bounds__(kThreads, 1)
                         const __grid_constant__ CUtensorMap tm_xhat,
                         const __grid_constant__ CUtensorMap tm_w,
                         const __grid_constant__ FusedParams p,
-                        const __grid_constant__ FusedBasis fb) {
+                        const __grid_constant__ FusedBasis fb,
+                        const __grid_constant__ FusedSchedule sc) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -170,7 +115,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   // scheduled as SMs free up; it waits for this grid before touching memory
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-  const int my_tiles = tiles_of_cta(p, cta, grid);
+  const int my_tiles = unit_tile_count(p, sc, cta, grid);
 
   if (warp == 0) {
     // =========================== TMA producer ===========================
@@ -184,7 +129,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       uint32_t it = 0;
       bool ok = true;
       for (int ti = 0; ti < my_tiles && ok && !p.test_stall; ++ti) {
-        const Tile tl = nth_tile(p, cta, grid, ti);
+        const WorkTile tl = unit_tile(p, sc, cta, grid, ti);
         const int bn = tl.is_gw ? p.BNw : p.BNx;
         const uint32_t tx = static_cast<uint32_t>(kABytes + bn * BK * 2);
         for (int kb = tl.kb0; kb < tl.kb0 + tl.n_kb; ++kb) {
@@ -223,7 +168,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       const uint32_t idesc_w = ptx::idesc_bf16(BM, p.BNw, true, true);
       const uint32_t idesc_x = ptx::idesc_bf16(BM, p.BNx, false, true);
       for (int ti = 0; ti < my_tiles && ok; ++ti) {
-        const Tile tl = nth_tile(p, cta, grid, ti);
+        const WorkTile tl = unit_tile(p, sc, cta, grid, ti);
         const int slot = ti & 1;
         const int n_kb = tl.n_kb;
         const uint32_t d_tmem = tmem_base + slot * kSlotCols;
@@ -272,7 +217,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     if (etid < kEStride) Eg[BM * kEStride + etid] = 0.f;
     named_bar_sync(bar_id, 128);
     for (int ti = 0; ti < my_tiles; ++ti) {
-      const Tile tl = nth_tile(p, cta, grid, ti);
+      const WorkTile tl = unit_tile(p, sc, cta, grid, ti);
       const int slot = ti & 1;
       const uint32_t uses = static_cast<uint32_t>(ti >> 1);
       const uint32_t acc_col = slot * kSlotCols;
@@ -313,6 +258,10 @@ __global__ void __launch_bounds__(kThreads, 1)
 }  // namespace fused
 
 // --------------------------------------------------------------- launcher ----
+static thread_local const FusedOverlap* g_overlap = nullptr;
+void set_fused_overlap(const FusedOverlap* ov) { g_overlap = ov; }
+const FusedOverlap* fused_overlap() { return g_overlap; }
+
 static thread_local bool g_test_stall = false;
 void set_test_stall(bool on) { g_test_stall = on; }
 bool test_stall() { return g_test_stall; }
@@ -325,7 +274,7 @@ bool fused_supported(const lbp_layer& L, const BasisPlan& bp) {
 }
 
 size_t fused_scratch_bytes(const lbp_layer& L, int r, FusedLayout* lay) {
-  const long long nb = static_cast<long long>(L.B) * (L.H / L.k) * (L.W / L.k);
+  const long long nb = static_cast<long long>(L.B) * blocks_along(L.H, L.k) * blocks_along(L.W, L.k);
   // Blocks per 128-row group.  With very few groups (low rank on a small token
   // grid) the expansion of a whole group, (128 / r) * k * k tokens per tile, falls
   // on a handful of CTAs: groups are then filled only partly (rows left zero)
@@ -366,9 +315,75 @@ size_t fused_scratch_bytes(const lbp_layer& L, int r, FusedLayout* lay) {
   return l.total;
 }
 
-int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void* g_W,
-                 const lbp_layer& L, const BasisPlan& bp, uint8_t* scratch, uint32_t* status,
-                 cudaStream_t stream, FusedPhaseHook hook, void* hook_arg) {
+// Expansion variant of a basis plan: 0 core butterfly, 1 4 x 4 core plus extra
+// bases, 2 8 x 8 core.
+static int epilogue_kind(const BasisPlan& bp) {
+  int n_outside = 0;
+  for (int q = 0; q < bp.r; ++q) n_outside += (bp.seq_i[q] >= 4 || bp.seq_j[q] >= 4) ? 1 : 0;
+  if (bp.LB == 8 && n_outside <= kFusedMaxExtra) return 1;
+  return bp.LB == 8 ? 2 : 0;
+}
+
+double fused_products_model_us(const lbp_layer& L, const BasisPlan& bp, int pairs) {
+  FusedLayout lay;
+  fused_scratch_bytes(L, bp.r, &lay);
+  PlanShape shape{};
+  shape.Cin = L.Cin;
+  shape.Cout = L.Cout;
+  shape.G = lay.G;
+  shape.bpt = lay.bpt;
+  shape.k = L.k;
+  shape.units = pairs;
+  shape.pair = 1;
+  shape.max_splits = static_cast<int>(lay.planes_bytes / (static_cast<size_t>(L.Cout) * L.Cin * 4));
+  shape.epi_kind = epilogue_kind(bp);
+  shape.num_kb_w = lay.G * 2;
+  shape.num_kb_x = (L.Cout + 63) / 64;
+  // measured times sit about a third above the model (the stages of a unit share
+  // its path to L2), plus the launch and the first operand tiles
+  return 1.35 * plan_products(shape).model_us + 4.0;
+}
+
+double fused_projection_model_us(const lbp_layer& L, const BasisPlan& bp, int ctas) {
+  const double T = static_cast<double>(L.B) * L.H * L.W;
+  const double nb = static_cast<double>(L.B) * blocks_along(L.H, L.k) * blocks_along(L.W, L.k);
+  const double bytes = 2.0 * (T + nb * bp.r) * (L.Cin + L.Cout);
+  // one SM streams about 70 GB/s through its tile ring; the chip about 5.2 TB/s
+  const double rate = ctas * 70e3 < 5.2e6 ? ctas * 70e3 : 5.2e6;   // bytes per microsecond
+  return bytes / rate + 5.0;
+}
+
+int fused_project(const void* x, const void* x_hat_dense, const void* g_y, const lbp_layer& L,
+                  const BasisPlan& bp, const FusedParams& p, uint32_t* status, cudaStream_t stream) {
+  const RowMap grouped{p.bpt, fused::BM};
+  const FusedOverlap* ov = fused_overlap();
+  cudaStream_t ps = ov != nullptr ? ov->proj_stream : stream;
+  if (ov != nullptr) set_projection_launch(ProjLaunch{ov->proj_ctas, ov->proj_ctas > 0, false});
+  int e = LBP_OK;
+  if (x_hat_dense == nullptr) {
+    e = launch_project2(g_y, p.gy_hat, L.Cout, x, p.x_hat, L.Cin, LBP_BF16, L.B, L.H, L.W, bp, grouped,
+                        status, ps, fused_scale_gy(L.k), fused_scale_x(L.k));
+  } else {
+    // x_hat was taken at forward time (Eq. 3), as orthonormal coefficients: it
+    // changes its row layout and its power-of-two scale
+    e = launch_regroup_rows(x_hat_dense, p.x_hat, p.nb, bp.r, grouped, L.Cin,
+                            fused_scale_x(L.k) * static_cast<float>(L.k), ps);
+    if (e == LBP_OK)
+      e = launch_project(g_y, p.gy_hat, LBP_BF16, L.B, L.H, L.W, L.Cout, bp, grouped, status, ps,
+                         fused_scale_gy(L.k));
+  }
+  if (ov != nullptr) {
+    set_projection_launch(ProjLaunch{0, false, true});
+    if (e != LBP_OK) return e;
+    LBP_CUDA_TRY(cudaEventRecord(ov->proj_done, ps));
+    LBP_CUDA_TRY(cudaStreamWaitEvent(stream, ov->proj_done, 0));
+  }
+  return e;
+}
+
+int launch_fused(const void* x, const void* x_hat_dense, const void* g_y, const void* W, void* g_x,
+                 void* g_W, const lbp_layer& L, const BasisPlan& bp, uint8_t* scratch,
+                 uint32_t* status, cudaStream_t stream, FusedPhaseHook hook, void* hook_arg) {
   using namespace fused;
   FusedLayout lay;
   fused_scratch_bytes(L, bp.r, &lay);
@@ -377,8 +392,8 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
   LBP_CUDA_TRY(cudaGetDevice(&dev));
   LBP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   FusedParams p{};
-  p.Hb = L.H / K;
-  p.Wb = L.W / K;
+  p.Hb = blocks_along(L.H, K);
+  p.Wb = blocks_along(L.W, K);
   p.nb = L.B * p.Hb * p.Wb;
   p.H = L.H;
   p.W = L.W;
@@ -388,7 +403,6 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
   p.Cin = L.Cin;
   p.Cout = L.Cout;
   p.gw_bf16 = L.gw_dtype == LBP_BF16 ? 1 : 0;
-  p.scale = 1.0f / static_cast<float>(K);
   p.x_hat = reinterpret_cast<__nv_bfloat16*>(scratch + lay.x_hat);
   p.gy_hat = reinterpret_cast<__nv_bfloat16*>(scratch + lay.gy_hat);
   p.gw_planes = reinterpret_cast<float*>(scratch + lay.planes);
@@ -433,120 +447,42 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
       for (int b = 0; b < bp.LB; ++b) fb.qmap[a * bp.LB + b] = bp.qmap[a * bp.LB + b];
   }
   if (fused_pair_supported(L, sms))
-    return launch_fused_pair(x, g_y, W, g_W, L, bp, p, fb, lay, sms, status, stream, hook, hook_arg);
+    return launch_fused_pair(x, x_hat_dense, g_y, W, g_W, L, bp, p, fb, lay, sms, status, stream, hook,
+                             hook_arg);
 
-  // Column tiles are multiples of 64 (one TMA chunk) up to 256.  Each
-  // candidate pair is scored by the operand bytes of the busiest CTA under the
-  // snake assignment of the tile list (the kernel is bound by operand traffic).
-  p.num_kb_x = (L.Cout + BK - 1) / BK;
+  // column tiles (multiples of one 64-wide TMA chunk, up to 256), K slices of g_W
+  // and the tile list of every CTA
   p.mt_w = (L.Cout + 127) / 128;
-  p.num_kb_w = p.G * (BM / BK);
-  const int cin64 = (L.Cin + 63) / 64 * 64;
   const int max_splits_by_ws =
       static_cast<int>(lay.planes_bytes / (static_cast<size_t>(L.Cout) * L.Cin * 4));
-  // the search costs tens of microseconds of host time: remember recent answers
-  struct PlanKey {
-    int Cin, Cout, G, sms, max_splits;
-    int BNw, BNx, splits, kbps;
-  };
-  static thread_local PlanKey plan_cache[16];
-  static thread_local int plan_cache_n = 0, plan_cache_next = 0;
-  bool cached = false;
-  for (int i = 0; i < plan_cache_n; ++i) {
-    const PlanKey& c = plan_cache[i];
-    if (c.Cin == L.Cin && c.Cout == L.Cout && c.G == p.G && c.sms == sms &&
-        c.max_splits == max_splits_by_ws) {
-      p.BNw = c.BNw;
-      p.BNx = c.BNx;
-      p.gw_splits = c.splits;
-      p.kb_per_split_w = c.kbps;
-      cached = true;
-      break;
-    }
-  }
-  if (!cached) {
-  double best = -1.0;
-  static const int kSplitChoices[] = {1, 2, 3, 4, 6, 8, 12, 16, 24, 32, 48, 64, 96, 128, 192};
-  for (int bnw = 64; bnw <= 256; bnw += 64) {
-    for (int bnx = 64; bnx <= 256; bnx += 64) {
-      if (bnw > cin64 || bnx > cin64) continue;
-      for (int want : kSplitChoices) {
-        if (want > 1 && (want > max_splits_by_ws || want > p.num_kb_w / 4)) continue;
-        const int kbps = (p.num_kb_w + want - 1) / want;
-        const int splits = (p.num_kb_w + kbps - 1) / kbps;
-        const int nt_w = (L.Cin + bnw - 1) / bnw, n_tx = (L.Cin + bnx - 1) / bnx;
-        const int n_gw = p.mt_w * nt_w * splits, n_gx = p.G * n_tx;
-        const double gw_cost = static_cast<double>(kbps) * (kABytes + bnw * 128.0) + 1500.0 * bnw;
-        const double gx_cost = static_cast<double>(p.num_kb_x) * (kABytes + bnx * 128.0) +
-                               6000.0 * bnx;   // plus the expansion of the tile
-        const int total = n_gw + n_gx;
-        const int grid = total < sms ? total : sms;
-        double worst = 0.0;
-        for (int c = 0; c < grid; ++c) {
-          double load = 0.0;
-          for (int round = 0; round * grid < total; ++round) {
-            const int t = round * grid + ((round & 1) ? grid - 1 - c : c);
-            if (t < total) load += t < n_gw ? gw_cost : gx_cost;
-          }
-          if (load > worst) worst = load;
-        }
-        if (splits > 1) {
-          // the reduce launch that follows: fixed cost plus its plane traffic at HBM
-          // speed, in the same unit (bytes a CTA ingests at ~100 GB/s)
-          const double plane_bytes = static_cast<double>(L.Cout) * L.Cin * 4.0;
-          worst += 600000.0 + (splits + 1.0) * plane_bytes / 40.0;
-        }
-        if (best < 0 || worst < best) {
-          best = worst;
-          p.BNw = bnw;
-          p.BNx = bnx;
-          p.gw_splits = splits;
-          p.kb_per_split_w = kbps;
-        }
-      }
-    }
-  }
-    PlanKey& c = plan_cache[plan_cache_next];
-    c = PlanKey{L.Cin, L.Cout, p.G, sms, max_splits_by_ws, p.BNw, p.BNx, p.gw_splits, p.kb_per_split_w};
-    plan_cache_next = (plan_cache_next + 1) % 16;
-    if (plan_cache_n < 16) ++plan_cache_n;
-  }
-  // tuning overrides: LBP_FUSED_TILES="BNw,BNx,splits"
-  if (tune_options().has_tiles) {
-    const int bw = tune_options().tiles_bnw, bx = tune_options().tiles_bnx,
-              sp = tune_options().tiles_splits;
-    if (bw >= 64 && bw <= 256 && bw % 64 == 0 &&
-        bx >= 64 && bx <= 256 && bx % 64 == 0 && sp >= 1 && (sp == 1 || sp <= max_splits_by_ws)) {
-      p.BNw = bw;
-      p.BNx = bx;
-      p.kb_per_split_w = (p.num_kb_w + sp - 1) / sp;
-      p.gw_splits = (p.num_kb_w + p.kb_per_split_w - 1) / p.kb_per_split_w;
-    }
-  }
-  if (tune_options().verbose)
-      fprintf(stderr, "lbp products: G=%d BNw=%d BNx=%d gw_splits=%d kb/split=%d\n", p.G, p.BNw, p.BNx,
-              p.gw_splits, p.kb_per_split_w);
+  PlanShape shape{};
+  shape.Cin = L.Cin;
+  shape.Cout = L.Cout;
+  shape.G = p.G;
+  shape.bpt = p.bpt;
+  shape.k = L.k;
+  shape.units = sms;
+  shape.pair = 0;
+  shape.max_splits = max_splits_by_ws;
+  shape.epi_kind = p.n_extra > 0 ? 1 : (p.lb_kernel == 8 ? 2 : 0);
+  shape.num_kb_w = p.num_kb_w;
+  shape.num_kb_x = p.num_kb_x;
+  const TilePlan& plan = plan_products(shape);
+  p.BNw = plan.BNw;
+  p.BNx = plan.BNx;
+  p.gw_splits = plan.splits;
+  p.kb_per_split_w = plan.kbps;
   p.n_tx = (L.Cin + p.BNx - 1) / p.BNx;
   p.nt_w = (L.Cin + p.BNw - 1) / p.BNw;
   p.n_gx_tiles = p.G * p.n_tx;
   p.n_gw_tiles = p.mt_w * p.nt_w * p.gw_splits;
-  p.gw_planes = reinterpret_cast<float*>(scratch + lay.planes);
-  p.gw_bf16 = L.gw_dtype == LBP_BF16 ? 1 : 0;
-  p.scale = 1.0f / static_cast<float>(K);
-  p.x_hat = reinterpret_cast<__nv_bfloat16*>(scratch + lay.x_hat);
-  p.gy_hat = reinterpret_cast<__nv_bfloat16*>(scratch + lay.gy_hat);
-  p.g_x = static_cast<__nv_bfloat16*>(g_x);
-  p.g_W = g_W;
-  p.status = status;
 #ifdef LBP_ROLE_TRACE
   p.trace = reinterpret_cast<unsigned long long*>(scratch + lay.trace);
   LBP_CUDA_TRY(cudaMemsetAsync(p.trace, 0, kFusedTraceBytes, stream));
 #endif
 
   // Algorithm 1, steps 1-2: x_hat and g_y_hat, rows padded to 128-row groups
-  if (int e = launch_project2(g_y, p.gy_hat, L.Cout, x, p.x_hat, L.Cin, LBP_BF16, L.B, L.H, L.W, bp,
-                              RowMap{p.bpt, BM}, status, stream))
-    return e;
+  if (int e = fused_project(x, x_hat_dense, g_y, L, bp, p, status, stream)) return e;
   if (hook != nullptr)
     if (int e = hook(hook_arg, stream)) return e;
 
@@ -572,7 +508,7 @@ int launch_fused(const void* x, const void* g_y, const void* W, void* g_x, void*
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    LBP_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tm_gyhat_k, tm_gyhat_mn, tm_xhat, tm_w, p, fb));
+    LBP_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tm_gyhat_k, tm_gyhat_mn, tm_xhat, tm_w, p, fb, plan.sched));
     count_launch();
     LBP_CUDA_TRY(cudaGetLastError());
     if (p.gw_splits > 1)

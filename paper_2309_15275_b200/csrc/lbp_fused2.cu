@@ -121,7 +121,7 @@ __device__ __forceinline__ void trace_mark(const FusedParams& p, int slot, bool 
   if (p.trace != nullptr) {
     unsigned long long now;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
-    unsigned long long* t = p.trace + blockIdx.x * 8 + slot;
+    unsigned long long* t = p.trace + blockIdx.x * kTraceSlots + slot;
     if (first_only) {
       if (*t == 0) *t = now;
     } else {
@@ -133,59 +133,6 @@ __device__ __forceinline__ void trace_mark(const FusedParams& p, int slot, bool 
 #endif
 }
 
-// ---- pair-tile list (same snake as the one-CTA kernel, over CTA pairs), taken
-// in list order ----
-struct PairTile {
-  int is_gw;
-  int a, b;        // GW: (i, j) ; GX: (group pair, n)
-  int kb0, n_kb;
-  int slice;
-};
-__device__ __forceinline__ int tiles_of_pair(const FusedParams& p, int pair, int pairs) {
-  const int total = p.n_gw_tiles + p.n_gx_tiles;
-  int n = 0;
-  for (int round = 0; round * pairs < total; ++round) {
-    const int pos = (round & 1) ? (pairs - 1 - pair) : pair;
-    if (round * pairs + pos < total) ++n;
-  }
-  return n;
-}
-__device__ __forceinline__ PairTile nth_pair_tile(const FusedParams& p, int pair, int pairs, int nth) {
-  const int total = p.n_gw_tiles + p.n_gx_tiles;
-  int seen = 0, id = 0;
-  for (int round = 0; round * pairs < total; ++round) {
-    const int pos = (round & 1) ? (pairs - 1 - pair) : pair;
-    const int t = round * pairs + pos;
-    if (t < total) {
-      if (seen == nth) {
-        id = t;
-        break;
-      }
-      ++seen;
-    }
-  }
-  PairTile tl;
-  if (id < p.n_gw_tiles) {
-    tl.is_gw = 1;
-    const int t = id / p.gw_splits;
-    tl.slice = id - t * p.gw_splits;
-    tl.a = t / p.nt_w;
-    tl.b = t - tl.a * p.nt_w;
-    tl.kb0 = tl.slice * p.kb_per_split_w;
-    const int end = tl.kb0 + p.kb_per_split_w;
-    tl.n_kb = (end < p.num_kb_w ? end : p.num_kb_w) - tl.kb0;
-  } else {
-    id -= p.n_gw_tiles;
-    tl.is_gw = 0;
-    tl.slice = 0;
-    tl.a = id / p.n_tx;
-    tl.b = id - tl.a * p.n_tx;
-    tl.kb0 = 0;
-    tl.n_kb = p.num_kb_x;
-  }
-  return tl;
-}
-
 // ------------------------------------------------------------------ kernel ----
 template <int K, int LB, int NEX = 0>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -194,7 +141,8 @@ __global__ void __launch_bounds__(kThreads, 1)
                              const __grid_constant__ CUtensorMap tm_xhat,
                              const __grid_constant__ CUtensorMap tm_w,
                              const __grid_constant__ FusedParams p,
-                             const __grid_constant__ FusedBasis fb) {
+                             const __grid_constant__ FusedBasis fb,
+                             const __grid_constant__ FusedSchedule sc) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -236,7 +184,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int my_tiles = tiles_of_pair(p, pair, pairs);
+  const int my_tiles = unit_tile_count(p, sc, pair, pairs);
   if (threadIdx.x == 0) trace_mark(p, 0);
   // the next kernel on the stream (the projection of the next call) may be
   // scheduled as SMs free up; it waits for this grid before touching memory
@@ -252,7 +200,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       uint32_t it = 0;
       bool ok = true;
       for (int ti = 0; ti < my_tiles && ok && !p.test_stall; ++ti) {
-        const PairTile tl = nth_pair_tile(p, pair, pairs, ti);
+        const WorkTile tl = unit_tile(p, sc, pair, pairs, ti);
         const int bn = tl.is_gw ? p.BNw : p.BNx;
         const int half = bn >> 1;
         const uint32_t tx_pair = 2u * static_cast<uint32_t>(kABytes + half * BK * 2);
@@ -294,7 +242,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       const uint32_t idesc_w = ptx::idesc_bf16(256, p.BNw, true, true);
       const uint32_t idesc_x = ptx::idesc_bf16(256, p.BNx, false, true);
       for (int ti = 0; ti < my_tiles && ok; ++ti) {
-        const PairTile tl = nth_pair_tile(p, pair, pairs, ti);
+        const WorkTile tl = unit_tile(p, sc, pair, pairs, ti);
         const int slot = ti & 1;
         const uint32_t d_tmem = tmem_base + slot * kSlotCols;
         const uint32_t idesc = tl.is_gw ? idesc_w : idesc_x;
@@ -309,6 +257,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             ok = false;
             break;
           }
+          if (kb == 0 && ti < 15) trace_mark(p, 8 + 8 * ti);
           ptx::tc_fence_after_sync();
           const uint32_t sa = ptx::smem_u32(smem + s * kStageBytes);
           const uint32_t sb = sa + kABytes;
@@ -324,6 +273,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
         if (!ok) break;
         mma_commit_pair(&acc_full[slot]);
+        if (ti < 15) trace_mark(p, 8 + 8 * ti + 1);
       }
       if (!ok) *abort_flag = 1;
       trace_mark(p, 3);
@@ -339,7 +289,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     if (etid < kEStride) Eg[BM * kEStride + etid] = 0.f;   // the zero row of the staging buffer
     fused::named_bar_sync(bar_id, 128);
     for (int ti = 0; ti < my_tiles; ++ti) {
-      const PairTile tl = nth_pair_tile(p, pair, pairs, ti);
+      const WorkTile tl = unit_tile(p, sc, pair, pairs, ti);
       const int slot = ti & 1;
       const uint32_t uses = static_cast<uint32_t>(ti >> 1);
       const bool ok = ptx::mbar_wait(&acc_full[slot], uses & 1u, p.status, (5u << 16) | 5u);
@@ -352,6 +302,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         break;
       }
       ptx::tc_fence_after_sync();
+      if (etid == 0 && ti < 15) trace_mark(p, 8 + 8 * ti + 2 + 2 * eg);
       fused::DrainTile dt;
       dt.is_gw = tl.is_gw;
       dt.bn = tl.is_gw ? p.BNw : p.BNx;
@@ -363,7 +314,14 @@ __global__ void __launch_bounds__(kThreads, 1)
       const uint32_t release_bar = map_to_rank(ptx::smem_u32(&acc_empty[slot]), 0);
       fused::drain_tile<K, LB, NEX>(p, fb, dt, Eg, bar_id, eg, etid, quarter, lane,
                                [release_bar]() { mbar_arrive_cluster(release_bar); });
-      if (etid == 0 && eg == 0) trace_mark(p, 5, true);
+      if (etid == 0 && ti < 15) {
+        trace_mark(p, 8 + 8 * ti + 3 + 2 * eg);
+#ifdef LBP_ROLE_TRACE
+        if (eg == 0 && p.trace != nullptr)
+          p.trace[blockIdx.x * kTraceSlots + 8 + 8 * ti + 6] =
+              (static_cast<unsigned long long>(tl.is_gw) << 32) | static_cast<unsigned>(tl.n_kb);
+#endif
+      }
     }
     if (etid == 0) trace_mark(p, 4);
   }
@@ -387,101 +345,41 @@ bool fused_pair_supported(const lbp_layer& L, int sms) {
 
 // `p` arrives with the geometry filled in (launch_fused); this chooses the
 // pair-tile shapes, launches the projection and then the pair kernel.
-int launch_fused_pair(const void* x, const void* g_y, const void* W, void* g_W, const lbp_layer& L,
+int launch_fused_pair(const void* x, const void* x_hat_dense, const void* g_y, const void* W,
+                      void* g_W, const lbp_layer& L,
                       const BasisPlan& bp, FusedParams p, const FusedBasis& fb,
                       const FusedLayout& lay, int sms, uint32_t* status, cudaStream_t stream,
                       FusedPhaseHook hook, void* hook_arg) {
   using namespace fused2;
-  const int pairs = sms / 2;
+  const FusedOverlap* ov = fused_overlap();
+  const int pairs = ov != nullptr && ov->prod_units > 0 && ov->prod_units < sms / 2 ? ov->prod_units
+                                                                                    : sms / 2;
   const int mt_w = (L.Cout + 255) / 256;    // 256 rows of g_W per pair-tile
   const int G2 = (p.G + 1) / 2;             // two row groups per GX pair-tile
   const int max_splits_by_ws =
       static_cast<int>(lay.planes_bytes / (static_cast<size_t>(L.Cout) * L.Cin * 4));
 
-  struct PlanKey {
-    int Cin, Cout, G, sms, max_splits;
-    int BNw, BNx, splits, kbps;
-  };
-  static thread_local PlanKey plan_cache[16];
-  static thread_local int plan_cache_n = 0, plan_cache_next = 0;
-  bool cached = false;
-  for (int i = 0; i < plan_cache_n; ++i) {
-    const PlanKey& c = plan_cache[i];
-    if (c.Cin == L.Cin && c.Cout == L.Cout && c.G == p.G && c.sms == sms &&
-        c.max_splits == max_splits_by_ws) {
-      p.BNw = c.BNw;
-      p.BNx = c.BNx;
-      p.gw_splits = c.splits;
-      p.kb_per_split_w = c.kbps;
-      cached = true;
-      break;
-    }
-  }
-  if (!cached) {
-    // per-CTA operand bytes of the busiest pair under the snake assignment
-    const int cin128 = (L.Cin + 127) / 128 * 128;
-    static const int kSplitChoices[] = {1, 2, 3, 4, 6, 8, 12, 16, 24, 32, 48, 64, 96, 128, 192};
-    double best = -1.0;
-    for (int bnw = 128; bnw <= 256; bnw += 128) {
-      for (int bnx = 128; bnx <= 256; bnx += 128) {
-        if (bnw > cin128 || bnx > cin128) continue;
-        for (int want : kSplitChoices) {
-          if (want > 1 && (want > max_splits_by_ws || want > p.num_kb_w / 4)) continue;
-          const int kbps = (p.num_kb_w + want - 1) / want;
-          const int splits = (p.num_kb_w + kbps - 1) / kbps;
-          const int nt_w = (L.Cin + bnw - 1) / bnw, n_tx = (L.Cin + bnx - 1) / bnx;
-          const int n_gw = mt_w * nt_w * splits, n_gx = G2 * n_tx;
-          const double gw_cost = static_cast<double>(kbps) * (kABytes + bnw * 64.0) + 1500.0 * bnw;
-          const double gx_cost =
-              static_cast<double>(p.num_kb_x) * (kABytes + bnx * 64.0) + 6000.0 * bnx;
-          const int total = n_gw + n_gx;
-          const int grid = total < pairs ? total : pairs;
-          double worst = 0.0;
-          for (int c = 0; c < grid; ++c) {
-            double load = 0.0;
-            for (int round = 0; round * grid < total; ++round) {
-              const int t = round * grid + ((round & 1) ? grid - 1 - c : c);
-              if (t < total) load += t < n_gw ? gw_cost : gx_cost;
-            }
-            if (load > worst) worst = load;
-          }
-          if (splits > 1) {
-            const double plane_bytes = static_cast<double>(L.Cout) * L.Cin * 4.0;
-            worst += 600000.0 + (splits + 1.0) * plane_bytes / 40.0;
-          }
-          if (best < 0 || worst < best) {
-            best = worst;
-            p.BNw = bnw;
-            p.BNx = bnx;
-            p.gw_splits = splits;
-            p.kb_per_split_w = kbps;
-          }
-        }
-      }
-    }
-    PlanKey& c = plan_cache[plan_cache_next];
-    c = PlanKey{L.Cin, L.Cout, p.G, sms, max_splits_by_ws, p.BNw, p.BNx, p.gw_splits, p.kb_per_split_w};
-    plan_cache_next = (plan_cache_next + 1) % 16;
-    if (plan_cache_n < 16) ++plan_cache_n;
-  }
-  if (tune_options().verbose)
-      fprintf(stderr, "lbp products (CTA pairs): G=%d BNw=%d BNx=%d gw_splits=%d kb/split=%d\n", p.G,
-              p.BNw, p.BNx, p.gw_splits, p.kb_per_split_w);
+  PlanShape shape{};
+  shape.Cin = L.Cin;
+  shape.Cout = L.Cout;
+  shape.G = p.G;
+  shape.bpt = p.bpt;
+  shape.k = L.k;
+  shape.units = pairs;
+  shape.pair = 1;
+  shape.max_splits = max_splits_by_ws;
+  shape.epi_kind = p.n_extra > 0 ? 1 : (p.lb_kernel == 8 ? 2 : 0);
+  shape.num_kb_w = p.num_kb_w;
+  shape.num_kb_x = p.num_kb_x;
+  const TilePlan& plan = plan_products(shape);
+  p.BNw = plan.BNw;
+  p.BNx = plan.BNx;
+  p.gw_splits = plan.splits;
+  p.kb_per_split_w = plan.kbps;
 #ifdef LBP_ROLE_TRACE
   p.trace = reinterpret_cast<unsigned long long*>(reinterpret_cast<uint8_t*>(p.x_hat) + lay.trace);
   LBP_CUDA_TRY(cudaMemsetAsync(p.trace, 0, kFusedTraceBytes, stream));
 #endif
-  if (tune_options().has_tiles) {   // tuning override "BNw,BNx,splits"
-    const int bw = tune_options().tiles_bnw, bx = tune_options().tiles_bnx,
-              sp = tune_options().tiles_splits;
-    if ((bw == 128 || bw == 256) &&
-        (bx == 128 || bx == 256) && sp >= 1 && (sp == 1 || sp <= max_splits_by_ws)) {
-      p.BNw = bw;
-      p.BNx = bx;
-      p.kb_per_split_w = (p.num_kb_w + sp - 1) / sp;
-      p.gw_splits = (p.num_kb_w + p.kb_per_split_w - 1) / p.kb_per_split_w;
-    }
-  }
   p.mt_w = mt_w;
   p.n_tx = (L.Cin + p.BNx - 1) / p.BNx;
   p.nt_w = (L.Cin + p.BNw - 1) / p.BNw;
@@ -489,9 +387,7 @@ int launch_fused_pair(const void* x, const void* g_y, const void* W, void* g_W, 
   p.n_gw_tiles = mt_w * p.nt_w * p.gw_splits;
 
   // Algorithm 1, steps 1-2: x_hat and g_y_hat, rows padded to 128-row groups
-  if (int e = launch_project2(g_y, p.gy_hat, L.Cout, x, p.x_hat, L.Cin, LBP_BF16, L.B, L.H, L.W, bp,
-                              RowMap{p.bpt, BM}, status, stream))
-    return e;
+  if (int e = fused_project(x, x_hat_dense, g_y, L, bp, p, status, stream)) return e;
   if (hook != nullptr)
     if (int e = hook(hook_arg, stream)) return e;
 
@@ -520,8 +416,11 @@ int launch_fused_pair(const void* x, const void* g_y, const void* W, void* g_W, 
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 2;
-    LBP_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tm_gyhat_k, tm_gyhat_mn, tm_xhat, tm_w, p, fb));
+    // Beside a projection on another stream the kernel is launched in plain stream
+    // order: launched early, its CTAs would sit on the SMs that projection is
+    // meant to get while they wait for the kernel ahead.
+    cfg.numAttrs = ov != nullptr ? 1 : 2;
+    LBP_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tm_gyhat_k, tm_gyhat_mn, tm_xhat, tm_w, p, fb, plan.sched));
     count_launch();
     LBP_CUDA_TRY(cudaGetLastError());
     if (p.gw_splits > 1)

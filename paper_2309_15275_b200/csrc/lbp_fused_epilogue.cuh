@@ -13,6 +13,8 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "lbp_fused.cuh"
 #include "ptx_sm100.cuh"
 #include "wht_device.cuh"
@@ -142,6 +144,22 @@ __device__ __forceinline__ void drain_tile(const FusedParams& p, const FusedBasi
     const int cc = etid % CPT, bs = etid / CPT;
     // element offsets of a token inside a block fit 32 bits (checked on the host)
     const int tok_stride = p.Cin, row_stride = p.W * p.Cin;
+    // first token of block bl of this group (channel 0) and how many of its K x K
+    // tokens lie on the grid
+    auto block_origin = [&](int bl, __nv_bfloat16** o, int* ulim, int* vlim) {
+      const int blk = m * p.bpt + bl;
+      const int bw = blk % p.Wb, t2 = blk / p.Wb, bh = t2 % p.Hb, b = t2 / p.Hb;
+      *o = p.g_x + ((static_cast<long long>(b) * p.H + bh * K) * p.W + bw * K) * p.Cin;
+      *ulim = p.H - bh * K < K ? p.H - bh * K : K;
+      *vlim = p.W - bw * K < K ? p.W - bw * K : K;
+    };
+    // the first block a thread expands is the same for every chunk of the tile
+    __nv_bfloat16* o_first = p.g_x;
+    int ulim_first = K, vlim_first = K;
+    if (bs < bg) {
+      block_origin(bs, &o_first, &ulim_first, &vlim_first);
+      o_first += t.col_base + cc * NCH;
+    }
     for (int c0 = eg * 32; c0 < t.bn; c0 += 32 * kEGroups) {
       uint32_t v[32];
       ptx::tmem_ld_32x32(t.tmem_acc + lane_bits + c0, v);
@@ -188,98 +206,119 @@ __device__ __forceinline__ void drain_tile(const FusedParams& p, const FusedBasi
           }
           hadamard_rows<LB, NCH>(acc);
           hadamard_cols<LB, NCH>(acc);
-          const int blk = m * p.bpt + bl;
-          const int bw = blk % p.Wb, t2 = blk / p.Wb, bh = t2 % p.Hb, b = t2 / p.Hb;
-          __nv_bfloat16* o = p.g_x +
-                             ((static_cast<long long>(b) * p.H + bh * K) * p.W + bw * K) * p.Cin + ch;
-          if constexpr (NEX > 0) {
-            // Bases outside the LB x LB core: B_{i,j}[u][v] = s_i(u) s_j(v) with
-            // s = +-1, so each adds +-coefficient to every token.  The row sign is
-            // folded into the coefficient once per token row, the column sign is
-            // a +-1.0 factor of an FMA.
-            static_assert(NCH == 4, "extras go with four channels per thread");
-            float ce[NEX][NCH];
-            uint32_t mu[NEX], mv[NEX];
+          __nv_bfloat16* o;
+          int ulim, vlim;
+          if (bl == bs) {
+            o = o_first + (ch - t.col_base - cc * NCH);
+            ulim = ulim_first;
+            vlim = vlim_first;
+          } else {
+            block_origin(bl, &o, &ulim, &vlim);
+            o += ch;
+          }
+          // Stores of one expanded block.  RAGGED: the block reaches past the grid
+          // (a side that is no multiple of K) and every token is checked; all other
+          // blocks take the unchecked form.  The 1/k of Eq. 7 is already in the
+          // coefficients (g_y_hat carries 1/k^2), so a value is rounded as it is.
+          auto emit = [&](auto ragged) {
+            constexpr bool RAGGED = decltype(ragged)::value;
+            if constexpr (NEX > 0) {
+              // Bases outside the LB x LB core: B_{i,j}[u][v] = s_i(u) s_j(v) with
+              // s = +-1, so each adds +-coefficient to every token.  The row sign is
+              // folded into the coefficient once per token row, the column sign is
+              // a +-1.0 factor of an FMA.
+              static_assert(NCH == 4, "extras go with four channels per thread");
+              float ce[NEX][NCH];
+              uint32_t mu[NEX], mv[NEX];
 #pragma unroll
-            for (int x = 0; x < NEX; ++x) {
-              const int q = fb.ex_q[x];
-              const int row_q = q >= 0 ? row_b + q : BM;
-              const float4 f =
-                  *reinterpret_cast<const float4*>(Eg + row_q * kEStride + ((cc ^ (row_q & 7)) << 2));
-              ce[x][0] = f.x;
-              ce[x][1] = f.y;
-              ce[x][2] = f.z;
-              ce[x][3] = f.w;
-              mu[x] = fb.ex_mu[x];
-              mv[x] = fb.ex_mv[x];
-            }
+              for (int x = 0; x < NEX; ++x) {
+                const int q = fb.ex_q[x];
+                const int row_q = q >= 0 ? row_b + q : BM;
+                const float4 f =
+                    *reinterpret_cast<const float4*>(Eg + row_q * kEStride + ((cc ^ (row_q & 7)) << 2));
+                ce[x][0] = f.x;
+                ce[x][1] = f.y;
+                ce[x][2] = f.z;
+                ce[x][3] = f.w;
+                mu[x] = fb.ex_mu[x];
+                mv[x] = fb.ex_mv[x];
+              }
 #pragma unroll
-            for (int a = 0; a < LB; ++a) {
+              for (int a = 0; a < LB; ++a) {
 #pragma unroll 1
-              for (int du = 0; du < RUN; ++du) {
-                const int u = a * RUN + du;
-                float ceu[NEX][NCH];
-#pragma unroll
-                for (int x = 0; x < NEX; ++x) {
-                  const float su = __uint_as_float(0x3f800000u | (((mu[x] >> u) & 1u) << 31));
-#pragma unroll
-                  for (int c = 0; c < NCH; ++c) ceu[x][c] = ce[x][c] * su;
-                }
-                __nv_bfloat16* orow = o + u * row_stride;
-#pragma unroll
-                for (int v = 0; v < K; ++v) {
-                  float val[NCH];
-#pragma unroll
-                  for (int c = 0; c < NCH; ++c) val[c] = acc[a][v / RUN][c];
+                for (int du = 0; du < RUN; ++du) {
+                  const int u = a * RUN + du;
+                  if (RAGGED && u >= ulim) break;
+                  float ceu[NEX][NCH];
 #pragma unroll
                   for (int x = 0; x < NEX; ++x) {
-                    const float sv = __uint_as_float(0x3f800000u | ((mv[x] << (31 - v)) & 0x80000000u));
+                    const float su = __uint_as_float(0x3f800000u | (((mu[x] >> u) & 1u) << 31));
 #pragma unroll
-                    for (int c = 0; c < NCH; ++c) val[c] = fmaf(sv, ceu[x][c], val[c]);
+                    for (int c = 0; c < NCH; ++c) ceu[x][c] = ce[x][c] * su;
                   }
-                  uint2 pk;
-                  pk.x = pack_bf16x2(val[0] * p.scale, val[1] * p.scale);
-                  pk.y = pack_bf16x2(val[2] * p.scale, val[3] * p.scale);
-                  *reinterpret_cast<uint2*>(orow + v * tok_stride) = pk;
+                  __nv_bfloat16* orow = o + u * row_stride;
+#pragma unroll
+                  for (int v = 0; v < K; ++v) {
+                    float val[NCH];
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) val[c] = acc[a][v / RUN][c];
+#pragma unroll
+                    for (int x = 0; x < NEX; ++x) {
+                      const float sv = __uint_as_float(0x3f800000u | ((mv[x] << (31 - v)) & 0x80000000u));
+#pragma unroll
+                      for (int c = 0; c < NCH; ++c) val[c] = fmaf(sv, ceu[x][c], val[c]);
+                    }
+                    uint2 pk;
+                    pk.x = pack_bf16x2(val[0], val[1]);
+                    pk.y = pack_bf16x2(val[2], val[3]);
+                    if (!RAGGED || v < vlim) *reinterpret_cast<uint2*>(orow + v * tok_stride) = pk;
+                  }
+                }
+              }
+            } else {
+              // each of the LB x LB values covers a RUN x RUN patch of tokens: round
+              // and pack once, store RUN * RUN times
+#pragma unroll
+              for (int a = 0; a < LB; ++a) {
+#pragma unroll
+                for (int b2 = 0; b2 < LB; ++b2) {
+                  if constexpr (NCH == 4) {
+                    uint2 pk;
+                    pk.x = pack_bf16x2(acc[a][b2][0], acc[a][b2][1]);
+                    pk.y = pack_bf16x2(acc[a][b2][2], acc[a][b2][3]);
+#pragma unroll
+                    for (int du = 0; du < RUN; ++du)
+#pragma unroll
+                      for (int dv = 0; dv < RUN; ++dv)
+                        if (!RAGGED || (a * RUN + du < ulim && b2 * RUN + dv < vlim))
+                          *reinterpret_cast<uint2*>(o + (a * RUN + du) * row_stride +
+                                                    (b2 * RUN + dv) * tok_stride) = pk;
+                  } else if constexpr (NCH == 1) {
+                    const __nv_bfloat16 hv = __float2bfloat16_rn(acc[a][b2][0]);
+#pragma unroll
+                    for (int du = 0; du < RUN; ++du)
+#pragma unroll
+                      for (int dv = 0; dv < RUN; ++dv)
+                        if (!RAGGED || (a * RUN + du < ulim && b2 * RUN + dv < vlim))
+                          o[(a * RUN + du) * row_stride + (b2 * RUN + dv) * tok_stride] = hv;
+                  } else {
+                    const uint32_t pk = pack_bf16x2(acc[a][b2][0], acc[a][b2][1]);
+#pragma unroll
+                    for (int du = 0; du < RUN; ++du)
+#pragma unroll
+                      for (int dv = 0; dv < RUN; ++dv)
+                        if (!RAGGED || (a * RUN + du < ulim && b2 * RUN + dv < vlim))
+                          *reinterpret_cast<uint32_t*>(o + (a * RUN + du) * row_stride +
+                                                       (b2 * RUN + dv) * tok_stride) = pk;
+                  }
                 }
               }
             }
-          } else {
-          // each of the LB x LB values covers a RUN x RUN patch of tokens: scale,
-          // round and pack once, store RUN * RUN times
-#pragma unroll
-          for (int a = 0; a < LB; ++a) {
-#pragma unroll
-            for (int b2 = 0; b2 < LB; ++b2) {
-              if constexpr (NCH == 4) {
-                uint2 pk;
-                pk.x = pack_bf16x2(acc[a][b2][0] * p.scale, acc[a][b2][1] * p.scale);
-                pk.y = pack_bf16x2(acc[a][b2][2] * p.scale, acc[a][b2][3] * p.scale);
-#pragma unroll
-                for (int du = 0; du < RUN; ++du)
-#pragma unroll
-                  for (int dv = 0; dv < RUN; ++dv)
-                    *reinterpret_cast<uint2*>(o + (a * RUN + du) * row_stride +
-                                              (b2 * RUN + dv) * tok_stride) = pk;
-              } else if constexpr (NCH == 1) {
-                const __nv_bfloat16 hv = __float2bfloat16_rn(acc[a][b2][0] * p.scale);
-#pragma unroll
-                for (int du = 0; du < RUN; ++du)
-#pragma unroll
-                  for (int dv = 0; dv < RUN; ++dv)
-                    o[(a * RUN + du) * row_stride + (b2 * RUN + dv) * tok_stride] = hv;
-              } else {
-                const uint32_t pk = pack_bf16x2(acc[a][b2][0] * p.scale, acc[a][b2][1] * p.scale);
-#pragma unroll
-                for (int du = 0; du < RUN; ++du)
-#pragma unroll
-                  for (int dv = 0; dv < RUN; ++dv)
-                    *reinterpret_cast<uint32_t*>(o + (a * RUN + du) * row_stride +
-                                                 (b2 * RUN + dv) * tok_stride) = pk;
-              }
-            }
-          }
-          }
+          };
+          if (ulim == K && vlim == K)
+            emit(std::false_type{});
+          else
+            emit(std::true_type{});
         }
       }
       named_bar_sync(bar_id, 128);

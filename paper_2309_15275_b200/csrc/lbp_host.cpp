@@ -23,6 +23,9 @@ void note_cuda_failure(cudaError_t e, const char* file, int line) {
 thread_local bool g_defer_wait = false;
 void set_projection_defer_wait(bool on) { g_defer_wait = on; }
 bool projection_defer_wait() { return g_defer_wait; }
+thread_local ProjLaunch g_proj_launch = {0, false, true};
+void set_projection_launch(ProjLaunch shape) { g_proj_launch = shape; }
+ProjLaunch projection_launch() { return g_proj_launch; }
 
 thread_local long long g_launches = 0;
 void count_launch(int n) { g_launches += n; }
@@ -120,6 +123,8 @@ void reload_tune_options() {
   e = std::getenv("LBP_FUSED_TILES");
   t.has_tiles = e != nullptr &&
                 std::sscanf(e, "%d,%d,%d", &t.tiles_bnw, &t.tiles_bnx, &t.tiles_splits) == 3;
+  e = std::getenv("LBP_BATCH_PROJ_SMS");
+  t.batch_proj_sms = e != nullptr ? std::atoi(e) : -1;
   g_tune = t;
   g_tune_loaded = true;
 }

@@ -53,6 +53,9 @@ int walsh_natural_index(int n, int s);
 int walsh_sign(int k, int s, int u);
 
 int check_order(int k);
+// Blocks along a grid side of n tokens: sides that are not multiples of k are
+// extended with zero tokens at their high end.
+inline int blocks_along(int n, int k) { return (n + k - 1) / k; }
 
 void set_last_cuda_error(cudaError_t e);
 void count_launch(int n = 1);   // bumps the per-thread kernel-launch counter
@@ -88,17 +91,34 @@ struct RowMap {
   int32_t tile_rows;
 };
 
+// `scale` multiplies the +-1 sums; 0 selects 1/k, the orthonormal coefficients of Eq. 6.
 int launch_project(const void* t, void* t_hat, int dtype, int B, int H, int W, int C,
-                   const BasisPlan& plan, RowMap rows, uint32_t* status, cudaStream_t stream);
+                   const BasisPlan& plan, RowMap rows, uint32_t* status, cudaStream_t stream,
+                   float scale = 0.f);
 
 // Per-thread switch read by the projection launchers (see ProjParams::defer_wait).
 void set_projection_defer_wait(bool on);
 bool projection_defer_wait();
 
+// Per-thread launch shape of the tensor-pipe projection kernels (set around a
+// launch by the side-stream mode of lbp_backward_batch):
+//   max_ctas      0 = one CTA per SM, else at most this many CTAs
+//   whole_tpcs    launch the CTAs as clusters of two, so that they fill both SMs
+//                 of a TPC and leave the other TPCs whole for the CTA pairs of a
+//                 products kernel that runs beside them
+//   programmatic  launch with programmatic stream serialization
+struct ProjLaunch {
+  int max_ctas;
+  bool whole_tpcs;
+  bool programmatic;
+};
+void set_projection_launch(ProjLaunch shape);
+ProjLaunch projection_launch();
+
 // Projects two tensors that share the token grid (x and g_y) in one launch.
 int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* out1, int C1,
                     int dtype, int B, int H, int W, const BasisPlan& plan, RowMap rows,
-                    uint32_t* status, cudaStream_t stream);
+                    uint32_t* status, cudaStream_t stream, float scale0 = 0.f, float scale1 = 0.f);
 
 // One-pass spectrum (bf16 data, k = 4 or 8): energy[i*k + j] of all k*k responses.
 // plan: all k*k pairs in raster order.
@@ -130,15 +150,37 @@ int launch_splitk_reduce(const float* planes, void* D, long long mn, int splits,
 
 int check_device_arch();
 
+// ---- kernels around Algorithm 1 (lbp_extras.cu) ----
+// g_W <- beta * g_W + a (+ b); a, b fp32 of mn elements, g_W fp32 or bf16.
+int launch_gw_combine(void* g_W, bool gw_bf16, const float* a, const float* b, float beta,
+                      long long mn, cudaStream_t stream);
+// Column sums in fp64 of n_sel selected rows of a (rows, C) matrix of `dtype`,
+// as bias_slabs(n_sel) partial rows of C doubles.  r == 0: rows 0..n_sel-1;
+// r > 0: the row of slot q of block i under the row map `rows`.
+int bias_slabs(long long n_sel);
+int launch_column_sum(const void* m, int dtype, long long n_sel, int C, RowMap rows, int r, int q,
+                      double* partial, cudaStream_t stream);
+// g_bias[c] <- beta * g_bias[c] + scale_a * (sum of the slabs of a) + (sum of the slabs of b)
+int launch_bias_finish(float* g_bias, int C, float beta, const double* a, int slabs_a, double scale_a,
+                       const double* b, int slabs_b, cudaStream_t stream);
+// Dense coefficient rows (blocks * r, C) -> rows padded to groups under `rows`
+// (rows no block owns are zero), every bf16 value multiplied by `factor` (a power of two).
+int launch_regroup_rows(const void* dense, void* grouped, int nb, int r, RowMap rows, int C,
+                        float factor, cudaStream_t stream);
+
 // Tuning switches, read from the environment once (first use):
 //   LBP_FUSED=0          separate product and expansion kernels instead of the
 //                        persistent products kernel
 //   LBP_PAIR=0           one-CTA products kernel also on wide layers
 //   LBP_FUSED_TILES=a,b,c  column tiles of the two products and K slices of g_W
 //   LBP_FUSED_VERBOSE=1  print the chosen tile plan
+//   LBP_BATCH_PROJ_SMS=n lbp_backward_batch: SMs given to the projection of the next
+//                        layer while the products kernel of a layer runs (0 = one
+//                        kernel at a time; unset = chosen per pair of layers)
 struct TuneOptions {
   bool fused, pair, verbose, has_tiles;
   int tiles_bnw, tiles_bnx, tiles_splits;
+  int batch_proj_sms;   // -1 = library default
 };
 const TuneOptions& tune_options();
 void reload_tune_options();   // test hook: read the environment again

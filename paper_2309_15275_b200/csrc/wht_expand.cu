@@ -71,6 +71,9 @@ __global__ void __launch_bounds__(256)
     // offset of token (u, v) of this block: tok0 + (u * W + v) * C
     const long long tok0 =
         ((static_cast<long long>(b) * p.H + bh * K) * p.W + bw * K) * p.C + c0;
+    // tokens of a last block that lie past the grid are not stored
+    const int ulim = p.H - bh * K < K ? p.H - bh * K : K;
+    const int vlim = p.W - bw * K < K ? p.W - bw * K : K;
 
     if constexpr (LB < 16) {
       constexpr int RUN = K / LB;
@@ -98,8 +101,9 @@ __global__ void __launch_bounds__(256)
         for (int u = 0; u < K; ++u) {
 #pragma unroll
           for (int v = 0; v < K; ++v) {
-            store_token<TO, OUT_BF16, NCH>(t, tok0 + (static_cast<long long>(u) * p.W + v) * p.C,
-                                           pass, acc[u / RUN][v / RUN], p.scale);
+            if (u < ulim && v < vlim)
+              store_token<TO, OUT_BF16, NCH>(t, tok0 + (static_cast<long long>(u) * p.W + v) * p.C,
+                                             pass, acc[u / RUN][v / RUN], p.scale);
           }
         }
       }
@@ -139,9 +143,10 @@ __global__ void __launch_bounds__(256)
 #pragma unroll
             for (int u = 0; u < 16; ++u) {
               const float v1[1] = {R[vh][u]};
-              store_token<TO, OUT_BF16, 1>(
-                  t, tok0 + (static_cast<long long>(u) * p.W + vh * 4 + v_lo) * p.C, pass, v1,
-                  p.scale);
+              if (u < ulim && vh * 4 + v_lo < vlim)
+                store_token<TO, OUT_BF16, 1>(
+                    t, tok0 + (static_cast<long long>(u) * p.W + vh * 4 + v_lo) * p.C, pass, v1,
+                    p.scale);
             }
           }
         }
@@ -195,8 +200,8 @@ int launch_expand(const void* t_hat, bool in_f32, void* t, int dtype, int B, int
                   const BasisPlan& bp, RowMap rows, cudaStream_t stream) {
   const int K = bp.k;
   ExpandParams p;
-  p.Hb = H / K;
-  p.Wb = W / K;
+  p.Hb = blocks_along(H, K);
+  p.Wb = blocks_along(W, K);
   p.nb = B * p.Hb * p.Wb;
   p.H = H;
   p.W = W;

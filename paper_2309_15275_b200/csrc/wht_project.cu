@@ -132,7 +132,7 @@ __global__ void __launch_bounds__(ProjCfg<K, sizeof(T) == 2>::kWarps * 32, 1)
 #pragma unroll
             for (int b = 0; b < LB; ++b) {
               const int q = plan.qmap[a * LB + b];
-              if (q >= 0) store_coeff<T, BF16, NCH>(out, row0 + q, C, c0, pass, acc[a][b], p.scale);
+              if (q >= 0) store_coeff<T, BF16, NCH>(out, row0 + q, C, c0, pass, acc[a][b], p.scale[which]);
             }
           }
         }
@@ -176,7 +176,7 @@ __global__ void __launch_bounds__(ProjCfg<K, sizeof(T) == 2>::kWarps * 32, 1)
                 const int q = plan.qmap[a * 16 + nh * 4 + n_lo];
                 if (q >= 0) {
                   const float v1[1] = {R[nh][a]};
-                  store_coeff<T, BF16, 1>(out, row0 + q, C, c0, pass, v1, p.scale);
+                  store_coeff<T, BF16, 1>(out, row0 + q, C, c0, pass, v1, p.scale[which]);
                 }
               }
             }
@@ -255,7 +255,7 @@ static int launch_t(const CUtensorMap* tmaps, T* out0, T* out1, const ProjParams
 
 int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* out1, int C1,
                     int dtype, int B, int H, int W, const BasisPlan& bp, RowMap rows,
-                    uint32_t* status, cudaStream_t stream) {
+                    uint32_t* status, cudaStream_t stream, float scale0, float scale1) {
   const int K = bp.k;
   const int es = dtype == LBP_BF16 ? 2 : 4;
   const int box_c = 128 / es;   // a box wider than C is legal: the excess is zero-filled
@@ -269,8 +269,8 @@ int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* ou
   }
 
   ProjParams p;
-  p.Hb = H / K;
-  p.Wb = W / K;
+  p.Hb = blocks_along(H, K);
+  p.Wb = blocks_along(W, K);
   p.nb = B * p.Hb * p.Wb;
   p.r = bp.r;
   p.bpt = rows.bpt;
@@ -285,7 +285,8 @@ int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* ou
   p.n_items0 = static_cast<uint32_t>(n0);
   p.n_items = static_cast<uint32_t>(n0 + n1);
   p.status = status;
-  p.scale = 1.0f / static_cast<float>(K);
+  p.scale[0] = scale0 > 0.f ? scale0 : 1.0f / static_cast<float>(K);
+  p.scale[1] = scale1 > 0.f ? scale1 : 1.0f / static_cast<float>(K);
   p.defer_wait = projection_defer_wait() ? 1 : 0;
 
   int dev = 0, sms = 0;
@@ -327,8 +328,10 @@ int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* ou
 }
 
 int launch_project(const void* t, void* t_hat, int dtype, int B, int H, int W, int C,
-                   const BasisPlan& bp, RowMap rows, uint32_t* status, cudaStream_t stream) {
-  return launch_project2(t, t_hat, C, nullptr, nullptr, 0, dtype, B, H, W, bp, rows, status, stream);
+                   const BasisPlan& bp, RowMap rows, uint32_t* status, cudaStream_t stream,
+                   float scale) {
+  return launch_project2(t, t_hat, C, nullptr, nullptr, 0, dtype, B, H, W, bp, rows, status, stream,
+                         scale, scale);
 }
 
 }  // namespace lbp

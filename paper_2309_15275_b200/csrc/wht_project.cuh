@@ -17,7 +17,9 @@ struct ProjParams {
   int32_t C[2], n_chunks[2];
   uint32_t n_items0, n_items;   // nb * n_chunks[0], nb * (n_chunks[0] + n_chunks[1])
   uint32_t* status;
-  float scale;                  // 1/k
+  // factor applied to the +-1 sums of tensor 0 / 1: 1/k gives the orthonormal
+  // coefficients of Eq. 6; the products kernel asks for other powers of two
+  float scale[2];
   // 0: wait for the preceding kernel on the stream before the first access;
   // 1: the caller vouches that nothing this kernel touches is touched by that
   // kernel, and the wait moves to the end (it then only keeps completion ordered)

@@ -123,6 +123,7 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
     const int blk = static_cast<int>(item / nch);
     const int chunk = static_cast<int>(item - blk * nch);
     const int C = p.C[which];
+    const float sc = p.scale[which];
     __nv_bfloat16* __restrict__ out = which ? out1 : out0;
     const uint32_t tile = ptx::smem_u32(my_tiles + s * Cfg::kTileBytes);
 
@@ -163,10 +164,10 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
         if (c < C) {   // C is a multiple of 8: a group of 8 channels is all in or all out
           if (q0 < p.r)
             ptx::st_global_hint_u32(out + (row0 + q0) * C + c,
-                                    pack_bf16x2(d[mt][nt][0] * p.scale, d[mt][nt][1] * p.scale), keep);
+                                    pack_bf16x2(d[mt][nt][0] * sc, d[mt][nt][1] * sc), keep);
           if (q1 < p.r)
             ptx::st_global_hint_u32(out + (row0 + q1) * C + c,
-                                    pack_bf16x2(d[mt][nt][2] * p.scale, d[mt][nt][3] * p.scale), keep);
+                                    pack_bf16x2(d[mt][nt][2] * sc, d[mt][nt][3] * sc), keep);
         }
       }
     }
@@ -280,6 +281,7 @@ __global__ void __launch_bounds__(kStripWarps * 32, 1)
     const int chunk = static_cast<int>(item - sg * nch);
     const uint32_t bw4 = sg % Wb4, t2 = sg / Wb4, bh = t2 % p.Hb, b = t2 / p.Hb;
     const int C = p.C[which];
+    const float sc = p.scale[which];
     __nv_bfloat16* __restrict__ out = which ? out1 : out0;
     const uint32_t tile = ptx::smem_u32(my_tiles + s * kStripTileBytes);
     const int cbase = chunk * 64 + 2 * tq;
@@ -312,10 +314,10 @@ __global__ void __launch_bounds__(kStripWarps * 32, 1)
           if (c < C) {
             if (q0 < p.r)
               ptx::st_global_hint_u32(out + (row0 + q0) * C + c,
-                                      pack_bf16x2(d[nt][0] * p.scale, d[nt][1] * p.scale), keep);
+                                      pack_bf16x2(d[nt][0] * sc, d[nt][1] * sc), keep);
             if (q1 < p.r)
               ptx::st_global_hint_u32(out + (row0 + q1) * C + c,
-                                      pack_bf16x2(d[nt][2] * p.scale, d[nt][3] * p.scale), keep);
+                                      pack_bf16x2(d[nt][2] * sc, d[nt][3] * sc), keep);
           }
         }
         // rows of a padded row tile that no block owns are kept at zero
@@ -339,22 +341,42 @@ __global__ void __launch_bounds__(kStripWarps * 32, 1)
   if (p.defer_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// Grid size and launch attributes of a projection launch under the per-thread
+// launch shape (see ProjLaunch).
+static int projection_grid(uint32_t want, int sms, cudaLaunchAttribute* attr, unsigned* n_attr) {
+  const ProjLaunch shape = projection_launch();
+  int cap = shape.max_ctas > 0 && shape.max_ctas < sms ? shape.max_ctas : sms;
+  int grid = static_cast<int>(want < static_cast<uint32_t>(cap) ? want : cap);
+  unsigned n = 0;
+  if (shape.programmatic) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  if (shape.whole_tpcs && grid >= 2) {
+    grid &= ~1;
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = 2;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  *n_attr = n;
+  return grid;
+}
+
 static int launch_strip4(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloat16* out1,
                          const ProjParams& p, const MmaPlan& mp, int sms, cudaStream_t stream) {
   auto kern = wht_project_mma_strip4_kernel;
   LBP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kStripSmemBytes));
   const uint32_t want = (p.n_items + kStripWarps - 1) / kStripWarps;
-  const int grid = static_cast<int>(want < static_cast<uint32_t>(sms) ? want : sms);
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(grid);
+  cudaLaunchAttribute attr[2];
+  cfg.gridDim = dim3(projection_grid(want, sms, attr, &cfg.numAttrs));
   cfg.blockDim = dim3(kStripWarps * 32);
   cfg.dynamicSmemBytes = kStripSmemBytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
   LBP_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmaps[0], tmaps[1], out0, out1, p, mp));
   count_launch();
   LBP_CUDA_TRY(cudaGetLastError());
@@ -384,17 +406,13 @@ static int launch_mma_one(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bf
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
   const uint32_t want = (p.n_items + Cfg::kWarps - 1) / Cfg::kWarps;
-  const int grid = static_cast<int>(want < static_cast<uint32_t>(sms) ? want : sms);
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(grid);
+  cudaLaunchAttribute attr[2];
+  cfg.gridDim = dim3(projection_grid(want, sms, attr, &cfg.numAttrs));
   cfg.blockDim = dim3(Cfg::kWarps * 32);
   cfg.dynamicSmemBytes = Cfg::kSmemBytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
   LBP_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmaps[0], tmaps[1], out0, out1, p, mp));
   count_launch();
   LBP_CUDA_TRY(cudaGetLastError());

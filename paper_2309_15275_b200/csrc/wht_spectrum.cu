@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
       }
   __syncthreads();
   // orthonormal coefficients: (1/k)^2 on the squares
-  const double s2 = static_cast<double>(p.scale) * static_cast<double>(p.scale);
+  const double s2 = static_cast<double>(p.scale[0]) * static_cast<double>(p.scale[0]);
   for (int i = threadIdx.x; i < R; i += NW * 32) atomicAdd(&energy[i], e_sm[i] * s2);
 }
 
@@ -296,7 +296,7 @@ __global__ void __launch_bounds__(MmaCfg<16>::kWarps * 32, 1)
         atomicAdd(&e_sm[sq.seq_of_nat[a] * K + sq.seq_of_nat[g + 8 * h]], static_cast<double>(v));
     }
   __syncthreads();
-  const double s2 = static_cast<double>(p.scale) * static_cast<double>(p.scale);
+  const double s2 = static_cast<double>(p.scale[0]) * static_cast<double>(p.scale[0]);
   for (int i = threadIdx.x; i < R; i += NW * 32) atomicAdd(&energy[i], e_sm[i] * s2);
 }
 
@@ -325,8 +325,8 @@ int launch_spectrum_mma(const void* t, int B, int H, int W, int C, const BasisPl
   CUtensorMap tmap;
   if (int e = encode_block_tensor_map(&tmap, t, LBP_BF16, B, H, W, C, K, 64, true)) return e;
   ProjParams p{};
-  p.Hb = H / K;
-  p.Wb = W / K;
+  p.Hb = blocks_along(H, K);
+  p.Wb = blocks_along(W, K);
   p.nb = B * p.Hb * p.Wb;
   p.r = K * K;
   p.bpt = 1;
@@ -337,7 +337,7 @@ int launch_spectrum_mma(const void* t, int B, int H, int W, int C, const BasisPl
   if (n0 >= (1ll << 31)) return LBP_ERR_SHAPE;
   p.n_items0 = p.n_items = static_cast<uint32_t>(n0);
   p.status = status;
-  p.scale = 1.0f / static_cast<float>(K);
+  p.scale[0] = p.scale[1] = 1.0f / static_cast<float>(K);
   MmaPlan mp;
   for (int q = 0; q < 64; ++q) {
     mp.nat_i[q] = q < bp.r ? bp.nat_i[q] : 0;

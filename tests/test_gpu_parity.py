@@ -127,8 +127,8 @@ def test_argument_errors_leave_outputs_untouched(dev):
         with pytest.raises(lbp.LbpError) as e:
             lbp.lbp_project(t, k, bases, out=out, ws=ws)
         assert e.value.status == status
-    with pytest.raises(lbp.LbpError) as e:      # W % k != 0
-        lbp.lbp_project(torch.zeros((1, 8, 12, 8), device=dev), 8, [(0, 0)], out=out, ws=ws)
+    with pytest.raises(lbp.LbpError) as e:      # an empty grid
+        lbp.lbp_project(torch.zeros((1, 0, 8, 8), device=dev), 8, [(0, 0)], out=out, ws=ws)
     assert e.value.status == 2
     with pytest.raises(lbp.LbpError) as e:      # C * 4 bytes not a multiple of 16
         lbp.lbp_project(torch.zeros((1, 8, 8, 6), device=dev), 8, [(0, 0)], out=out, ws=ws)
@@ -367,7 +367,7 @@ def test_spectrum_argument_errors(dev):
         lbp.lbp_spectrum(t, 8, out=e, ws=torch.zeros(256, dtype=torch.uint8, device=dev))
     assert err.value.status == 7 and float(e.min()) == -1.0
     with pytest.raises(ValueError):
-        lbp.lbp_spectrum(torch.zeros((1, 8, 12, 64), dtype=torch.bfloat16, device=dev), 8)
+        lbp.lbp_spectrum(torch.zeros((1, 8, 12, 60), dtype=torch.bfloat16, device=dev), 8)
 
 
 # ------------------------------------------------ autograd front end ----

@@ -79,7 +79,10 @@ def test_workspace_bytes():
     rows = 512 * 8
     assert n8 >= rows * (768 + 3072) * 2 + rows * 768 * 4
     assert n16 > n8
-    assert lbp.lbp_workspace_bytes(128, 16, 12, 768, 3072, 8, lbp.LBP_BF16, lbp.LBP_F32, 8) == 0   # W % k
+    # a grid side that is no multiple of k is extended with zero tokens: as many blocks as 16 x 16
+    assert (lbp.lbp_workspace_bytes(128, 16, 12, 768, 3072, 8, lbp.LBP_BF16, lbp.LBP_F32, 8)
+            == lbp.lbp_workspace_bytes(128, 16, 16, 768, 3072, 8, lbp.LBP_BF16, lbp.LBP_F32, 8))
+    assert lbp.lbp_workspace_bytes(128, 16, 0, 768, 3072, 8, lbp.LBP_BF16, lbp.LBP_F32, 8) == 0
     assert lbp.lbp_workspace_bytes(128, 16, 16, 768, 3072, 8, lbp.LBP_F32, lbp.LBP_BF16, 8) == 0   # dtype combo
     assert lbp.lbp_workspace_bytes(128, 16, 16, 768, 3072, 8, lbp.LBP_BF16, lbp.LBP_F32, 65) == 0
 
@@ -119,7 +122,9 @@ def test_select_lhe_argument_errors():
         lbp.lbp_select_lhe(np.ones((5, 5)), 5, 3)
     assert err.value.status == 3
     assert lbp.lbp_spectrum_workspace_bytes(2, 16, 16, 64, 8, lbp.LBP_BF16) >= 2 * 16 * 16 * 64 * 2
-    assert lbp.lbp_spectrum_workspace_bytes(2, 15, 16, 64, 8, lbp.LBP_BF16) == 0
+    assert (lbp.lbp_spectrum_workspace_bytes(2, 15, 16, 64, 8, lbp.LBP_BF16)
+            == lbp.lbp_spectrum_workspace_bytes(2, 16, 16, 64, 8, lbp.LBP_BF16))
+    assert lbp.lbp_spectrum_workspace_bytes(2, 15, 16, 60, 8, lbp.LBP_BF16) == 0
 
 
 def test_batch_arguments_are_checked_on_the_host_before_any_device_call():
@@ -164,3 +169,35 @@ def test_batch_arguments_are_checked_on_the_host_before_any_device_call():
     assert lib.lbp_backward_batch(0, arr(x), arr(gy), arr(w), arr(gx), arr(gw), lays,
                                   b._bases(bases), r, arr(ws), (ctypes.c_size_t * n)(*need), None, None) == 2
     assert "overlap" in lbp.lbp_status_string(12)
+
+
+@pytest.mark.parametrize("Cin,Cout,G,bpt,units,pair", [
+    (768, 2304, 32, 16, 74, 1), (768, 768, 32, 16, 74, 1), (768, 3072, 32, 16, 74, 1),
+    (3072, 768, 32, 16, 74, 1), (1024, 4096, 25, 21, 74, 1), (48, 192, 196, 16, 148, 0),
+    (192, 48, 196, 16, 148, 0), (64, 64, 1, 4, 148, 0), (768, 3072, 5, 2, 66, 1)])
+def test_tile_plan_covers_every_tile_once(Cin, Cout, G, bpt, units, pair):
+    # what the products kernel is told to do: every tile of both products exactly
+    # once, GX tiles (long epilogue) ahead of GW tiles on every unit
+    max_splits = 8
+    info, lists = lbp.lbp_test_tile_plan(Cin, Cout, G, bpt, 8, units, pair, max_splits)
+    row_tile = 256 if pair else 128
+    step = 128 if pair else 64
+    assert info["BNw"] % step == 0 and info["BNx"] % step == 0 and info["BNw"] <= 256 and info["BNx"] <= 256
+    assert 1 <= info["splits"] <= max_splits
+    assert info["kbps"] * info["splits"] >= 2 * G > info["kbps"] * (info["splits"] - 1)
+    n_gw = -(-Cout // row_tile) * -(-Cin // info["BNw"]) * info["splits"]
+    n_gx = (-(-G // 2) if pair else G) * -(-Cin // info["BNx"])
+    assert info["listed"] and lists is not None
+    flat = [t for unit in lists for t in unit]
+    assert sorted(flat) == list(range(n_gw + n_gx))
+    for unit in lists:
+        kinds = [t < n_gw for t in unit]            # True = GW
+        assert kinds == sorted(kinds)               # all GX tiles first
+    # no unit is left without work while another holds three tiles more
+    sizes = [len(u) for u in lists[:min(units, n_gw + n_gx)]]
+    assert min(sizes) >= 1
+
+
+def test_tile_plan_without_a_table_for_very_many_tiles():
+    info, lists = lbp.lbp_test_tile_plan(3072, 768, 400, 16, 8, 74, 1, 1)
+    assert not info["listed"] and lists is None
