@@ -176,9 +176,19 @@ int lbp_backward(const void* x, const void* g_y, const void* W,
  * ws_bytes[i]) and gives bit-identical results.  x .. ws, ws_bytes: host arrays
  * of n entries.  What one problem writes (g_x, g_W, ws) no other problem may
  * read or write (LBP_ERR_OVERLAP); inputs may be shared.  Knowing that, the
- * library lets the projection kernel of problem i + 1 start on the SMs that the
- * products kernel of problem i has already left instead of waiting for its last
- * tile.  done_events: NULL, or a host array of n cudaEvent_t handles (as void*,
+ * library overlaps the problems:
+ *  - bf16 problems of rank <= 16 on wide layers: the projections run on a
+ *    stream of the library's own (one non-blocking stream and a set of events
+ *    per device, created at the first such call on that device and kept: make
+ *    that call outside any stream capture), the projection of one problem on
+ *    part of the SMs beside the products kernel of another on the rest; the
+ *    problems are taken in the order that leaves least of it exposed, not
+ *    necessarily the given one.  Everything is ordered behind what `stream` held
+ *    at the call, and `stream` ends up behind all of it.
+ *  - otherwise the projection kernel of problem i + 1 starts on the SMs that the
+ *    products kernel of problem i has already left instead of waiting for its
+ *    last tile.
+ * done_events: NULL, or a host array of n cudaEvent_t handles (as void*,
  * an entry may be NULL): event i is recorded on `stream` behind the last kernel
  * of problem i, so that the caller can start what consumes g_W[i] / g_x[i] on
  * another stream (the data-parallel all-reduce of g_W, the one exchange step

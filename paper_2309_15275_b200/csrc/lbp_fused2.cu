@@ -46,7 +46,18 @@ constexpr int kABytes = BM * BK * 2;             // 16 KB: this CTA's 128 rows o
 constexpr int kBBytes = 128 * BK * 2;            // 16 KB: this CTA's half of B (up to 128 columns)
 constexpr int kStageBytes = kABytes + kBBytes;   // 32 KB
 constexpr int kChunkBytes = 64 * BK * 2;
-constexpr int kThreads = (2 + 4 * kEGroups) * 32;
+// warps 0-3: TMA producer, tensor-core issuer, two spare; then kEGroups epilogue
+// groups of four warps, each a warpgroup of its own (register reallocation below)
+constexpr int kThreads = (4 + 4 * kEGroups) * 32;
+// Registers per thread once the roles have parted (setmaxnreg).  The launch
+// gives each of the three warpgroups 128 x 168 registers; the first keeps
+// kRegsFeed per thread, the two epilogue warpgroups grow to kRegsEpilogue.  The
+// shares must add up to exactly what the block was launched with: a larger sum
+// would leave the last warpgroup waiting for registers that never come.
+constexpr int kRegsFeed = 104;
+constexpr int kRegsEpilogue = 200;
+static_assert(kEGroups == 2 && kRegsFeed + kEGroups * kRegsEpilogue == (1 + kEGroups) * 168,
+              "register split must add up to what the block was launched with");
 constexpr int kOffE = kStages * kStageBytes;
 constexpr int kOffBar = kOffE + kEGroups * kEBytes;
 constexpr int kSmemBytes = kOffBar + 256 + 1024;
@@ -190,6 +201,11 @@ __global__ void __launch_bounds__(kThreads, 1)
   // scheduled as SMs free up; it waits for this grid before touching memory
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+  // The roles part here, and with them the registers: the first warpgroup gives
+  // up what it does not need, the epilogue warpgroups take it (the expansion
+  // holds a whole coefficient array per thread).
+  if (warp < 4) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsFeed));
   if (warp == 0) {
     // =========================== TMA producer (both CTAs) ===========================
     if (ptx::elect_one()) {
@@ -278,10 +294,12 @@ __global__ void __launch_bounds__(kThreads, 1)
       if (!ok) *abort_flag = 1;
       trace_mark(p, 3);
     }
+  }
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsEpilogue));
     // =========================== epilogue (both CTAs, own 128 rows) ===========================
-    const int eg = (warp - 2) >> 2;
-    const int ew = (warp - 2) & 3;
+    const int eg = (warp - 4) >> 2;
+    const int ew = (warp - 4) & 3;
     const int quarter = warp & 3;
     const int etid = ew * 32 + lane;
     float* const Eg = E + eg * (kEBytes / 4);

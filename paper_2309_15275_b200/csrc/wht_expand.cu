@@ -97,13 +97,24 @@ __global__ void __launch_bounds__(256)
         }
         hadamard_rows<LB, NCH>(acc);
         hadamard_cols<LB, NCH>(acc);
+        if (ulim == K && vlim == K) {
 #pragma unroll
-        for (int u = 0; u < K; ++u) {
+          for (int u = 0; u < K; ++u) {
 #pragma unroll
-          for (int v = 0; v < K; ++v) {
-            if (u < ulim && v < vlim)
+            for (int v = 0; v < K; ++v) {
               store_token<TO, OUT_BF16, NCH>(t, tok0 + (static_cast<long long>(u) * p.W + v) * p.C,
                                              pass, acc[u / RUN][v / RUN], p.scale);
+            }
+          }
+        } else {   // a block that reaches past the grid: every token is checked
+#pragma unroll
+          for (int u = 0; u < K; ++u) {
+#pragma unroll
+            for (int v = 0; v < K; ++v) {
+              if (u < ulim && v < vlim)
+                store_token<TO, OUT_BF16, NCH>(t, tok0 + (static_cast<long long>(u) * p.W + v) * p.C,
+                                               pass, acc[u / RUN][v / RUN], p.scale);
+            }
           }
         }
       }

@@ -127,9 +127,9 @@ def test_argument_errors_leave_outputs_untouched(dev):
         with pytest.raises(lbp.LbpError) as e:
             lbp.lbp_project(t, k, bases, out=out, ws=ws)
         assert e.value.status == status
-    with pytest.raises(lbp.LbpError) as e:      # an empty grid
+    with pytest.raises(lbp.LbpError) as e:      # an empty grid (no storage: a null pointer, too)
         lbp.lbp_project(torch.zeros((1, 0, 8, 8), device=dev), 8, [(0, 0)], out=out, ws=ws)
-    assert e.value.status == 2
+    assert e.value.status in (1, 2)
     with pytest.raises(lbp.LbpError) as e:      # C * 4 bytes not a multiple of 16
         lbp.lbp_project(torch.zeros((1, 8, 8, 6), device=dev), 8, [(0, 0)], out=out, ws=ws)
     assert e.value.status == 6
