@@ -244,7 +244,7 @@ def run_gpu(args):
     import torch.distributed as dist
     import paper_2309_15275_b200 as lbp
     import synth
-    from paper_2309_15275_b200.dist import allreduce_gw
+    from paper_2309_15275_b200.dist import GwReducer, allreduce_gw
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -288,9 +288,7 @@ def run_gpu(args):
     # stream as soon as that layer's kernels are done (an event per layer recorded by
     # the batch call), under the kernels of the layers that follow.
     cur = torch.cuda.current_stream()
-    comm = torch.cuda.Stream(device=dev) if world > 1 else None
-    done_ev = [torch.cuda.Event() for _ in layers] if world > 1 else None
-    comm_ev = torch.cuda.Event() if world > 1 else None
+    reducer = GwReducer(len(layers), dev)
 
     def step(wss=None, bases_=bases):
         # the four layers are independent problems with their own buffers: one call
@@ -298,14 +296,8 @@ def run_gpu(args):
                                [L["w"] for L in layers], k, bases_,
                                g_xs=[L["gx"] for L in layers], g_Ws=[L["gw"] for L in layers],
                                wss=wss if wss is not None else [L["ws"] for L in layers],
-                               done_events=done_ev)
-        if world > 1:
-            with torch.cuda.stream(comm):
-                for L, e in zip(layers, done_ev):
-                    comm.wait_event(e)
-                    allreduce_gw(L["gw"])
-                comm_ev.record(comm)
-            cur.wait_event(comm_ev)        # the step ends when every g_W is summed
+                               done_events=reducer.events())
+        reducer.reduce([L["gw"] for L in layers])
 
     def barrier():
         if world > 1:

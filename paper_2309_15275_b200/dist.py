@@ -26,3 +26,50 @@ def allreduce_gw(g_W: torch.Tensor) -> torch.Tensor:
     if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
         dist.all_reduce(g_W, op=dist.ReduceOp.SUM)
     return g_W
+
+
+class GwReducer:
+    """Sums the g_W of several layers over the ranks while later layers still
+    compute: the all-reduce of layer i is issued as soon as that layer's kernels
+    are done, not after the whole batch call.
+
+    On GPUs the reductions run on a stream of their own, each behind the event
+    that lbp_backward_batch records for its layer (`events()` is what to pass as
+    `done_events`); `reduce()` enqueues them and makes the current stream wait
+    for the last one.  On CPU tensors (gloo) the reductions are started together
+    as asynchronous operations and waited for in order.  The sums are the same as
+    with one blocking all-reduce per layer after the call."""
+
+    def __init__(self, n_layers: int, device=None):
+        self.n = n_layers
+        self.active = dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1
+        self.cuda = self.active and device is not None and torch.device(device).type == "cuda"
+        if self.cuda:
+            self.stream = torch.cuda.Stream(device=device)
+            self._events = [torch.cuda.Event() for _ in range(n_layers)]
+            self._joined = torch.cuda.Event()
+        else:
+            self.stream, self._events, self._joined = None, None, None
+
+    def events(self):
+        """Events for lbp_backward_batch(done_events=...), or None when nothing is reduced."""
+        return self._events
+
+    def reduce(self, g_Ws):
+        if not self.active:
+            return g_Ws
+        if len(g_Ws) != self.n:
+            raise ValueError("one g_W per layer")
+        if self.cuda:
+            cur = torch.cuda.current_stream()
+            with torch.cuda.stream(self.stream):
+                for g, e in zip(g_Ws, self._events):
+                    self.stream.wait_event(e)
+                    dist.all_reduce(g, op=dist.ReduceOp.SUM)
+                self._joined.record(self.stream)
+            cur.wait_event(self._joined)          # the step ends when every g_W is summed
+        else:
+            handles = [dist.all_reduce(g, op=dist.ReduceOp.SUM, async_op=True) for g in g_Ws]
+            for h in handles:
+                h.wait()
+        return g_Ws

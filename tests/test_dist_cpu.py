@@ -10,7 +10,7 @@ import torch.distributed as dist
 import torch.multiprocessing as mp
 
 from oracle import lbp_oracle as O
-from paper_2309_15275_b200.dist import allreduce_gw, shard_images
+from paper_2309_15275_b200.dist import GwReducer, allreduce_gw, shard_images
 
 
 def _free_port():
@@ -45,6 +45,38 @@ def test_sharded_gw_allreduce_matches_full_batch(tmp_path):
     mp.spawn(_worker, args=(world, _free_port(), B, str(tmp_path)), nprocs=world, join=True)
     for r in range(world):
         assert (tmp_path / f"rank{r}.txt").read_text() == "ok"
+
+
+def _reducer_worker(rank, world, port, out_dir):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    rng = np.random.default_rng(11 + rank)
+    shapes = [(5, 6), (3, 3), (8, 2), (1, 7)]
+    mine = [torch.from_numpy(rng.standard_normal(s)) for s in shapes]
+    serial = [t.clone() for t in mine]
+    for t in serial:                      # one blocking all-reduce per layer, after the call
+        allreduce_gw(t)
+    red = GwReducer(len(shapes))          # issued together, as the layers finish
+    assert red.events() is None           # no device: nothing to record
+    red.reduce(mine)
+    ok = all(torch.equal(a, b) for a, b in zip(mine, serial))
+    with open(os.path.join(out_dir, f"red{rank}.txt"), "w") as f:
+        f.write("ok" if ok else "mismatch")
+    dist.destroy_process_group()
+
+
+def test_overlapped_gw_reduction_equals_the_serial_form(tmp_path):
+    world = 2
+    mp.spawn(_reducer_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    for r in range(world):
+        assert (tmp_path / f"red{r}.txt").read_text() == "ok"
+
+
+def test_reducer_is_a_noop_on_one_rank():
+    red = GwReducer(2)
+    t = [torch.ones(3), torch.ones(2)]
+    assert red.events() is None and red.reduce(t) is t and torch.equal(t[0], torch.ones(3))
 
 
 def test_shard_images_partition():
