@@ -54,7 +54,7 @@ def _peaks():
 # DRAM traffic per step (sum over the four layers, bytes) of the two kernels, from
 # the ncu capture summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum);
 # None = not captured for the current kernels.
-NCU_TRAFFIC_PER_STEP = {"wht_project_mma_kernel": None, "lbp_products_pair_kernel": None}
+NCU_TRAFFIC_PER_STEP = {"wht_project_mma_kernel": 828.9e6, "lbp_products_pair_kernel": 299.6e6}
 
 
 # ------------------------------------------------------------------ clocks ----
