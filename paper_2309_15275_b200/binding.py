@@ -430,7 +430,7 @@ def lbp_backward_projected(x_hat, g_y, W, k: int, bases, *, gw_dtype: torch.dtyp
     _check(_lib().lbp_backward_projected(_dev(x_hat, "x_hat"), _dev(g_y, "g_y"), _dev(W, "W"),
                                          _dev(g_x, "g_x"), _dev(g_W, "g_W"), C.byref(lay),
                                          _bases(bases), r, _dev(ws, "ws"), ws.numel(), _stream()),
-           "lbp_backward_projected", "lbp_test_tile_plan")
+           "lbp_backward_projected")
     return g_x, g_W
 
 
