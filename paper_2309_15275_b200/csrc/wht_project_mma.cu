@@ -24,6 +24,81 @@
 
 namespace lbp {
 
+// Where a warp is in its list of items (item = one block x one 64-channel
+// chunk of one of the two tensors; a warp takes every `stride`-th item).  The
+// position is decoded with divisions once, then moved by precomputed steps with
+// carries: a handful of additions per item where the divisions cost a third of
+// the warp's instructions.
+struct ItemSteps {
+  uint32_t chunk, blk, bw, bh, b, grp, j;   // `stride` items, as steps of each coordinate
+};
+struct ItemCursor {
+  uint32_t item;               // index over both tensors
+  uint32_t which;              // 0 / 1: tensor
+  uint32_t chunk, blk;         // 64-channel chunk, block
+  uint32_t bw, bh, b;          // block coordinates on the grid
+  uint32_t grp, j;             // row group and place inside it: blk = grp * bpt + j
+
+  __device__ __forceinline__ void decode(const ProjParams& p, uint32_t it) {
+    item = it;
+    which = it >= p.n_items0 ? 1u : 0u;
+    const uint32_t local = it - (which ? p.n_items0 : 0u);
+    const uint32_t nch = static_cast<uint32_t>(p.n_chunks[which]);
+    blk = local / nch;
+    chunk = local - blk * nch;
+    bw = blk % p.Wb;
+    const uint32_t t2 = blk / p.Wb;
+    bh = t2 % p.Hb;
+    b = t2 / p.Hb;
+    grp = blk / p.bpt;
+    j = blk - grp * p.bpt;
+  }
+  static __device__ __forceinline__ ItemSteps steps(const ProjParams& p, uint32_t stride, int w) {
+    ItemSteps s;
+    const uint32_t nch = static_cast<uint32_t>(p.n_chunks[w]);
+    s.blk = stride / nch;
+    s.chunk = stride - s.blk * nch;
+    s.bw = s.blk % p.Wb;
+    const uint32_t t2 = s.blk / p.Wb;
+    s.bh = t2 % p.Hb;
+    s.b = t2 / p.Hb;
+    s.grp = s.blk / p.bpt;
+    s.j = s.blk - s.grp * p.bpt;
+    return s;
+  }
+  // `stride` items further; st = the steps of the tensor the cursor is in
+  __device__ __forceinline__ void advance(const ProjParams& p, uint32_t stride, const ItemSteps& st) {
+    const uint32_t next = item + stride;
+    if (which == 0u && next >= p.n_items0) {   // into the second tensor: once per warp
+      decode(p, next);
+      return;
+    }
+    item = next;
+    const uint32_t nch = static_cast<uint32_t>(p.n_chunks[which]);
+    chunk += st.chunk;
+    const uint32_t carry = chunk >= nch ? 1u : 0u;
+    chunk -= carry ? nch : 0u;
+    blk += st.blk + carry;
+    bw += st.bw + carry;
+    if (bw >= static_cast<uint32_t>(p.Wb)) {
+      bw -= p.Wb;
+      bh += 1u;
+    }
+    bh += st.bh;
+    if (bh >= static_cast<uint32_t>(p.Hb)) {
+      bh -= p.Hb;
+      b += 1u;
+    }
+    b += st.b;
+    j += st.j + carry;
+    if (j >= static_cast<uint32_t>(p.bpt)) {
+      j -= p.bpt;
+      grp += 1u;
+    }
+    grp += st.grp;
+  }
+};
+
 template <int K, int MT>
 __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
     wht_project_mma_kernel(const __grid_constant__ CUtensorMap tmap0,
@@ -73,19 +148,21 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
   // the coefficients are read back from L2 by the kernel that follows
   const uint64_t keep = ptx::l2_policy_evict_last();
 
-  auto issue = [&](uint32_t idx, int s) {
-    uint32_t item = first + idx * stride;
-    const int which = item >= p.n_items0;
-    if (which) item -= p.n_items0;
-    const uint32_t nch = static_cast<uint32_t>(p.n_chunks[which]);
-    const uint32_t blk = item / nch, chunk = item - blk * nch;
-    const uint32_t bw = blk % p.Wb, t2 = blk / p.Wb, bh = t2 % p.Hb, b = t2 / p.Hb;
+  const ItemSteps steps0 = ItemCursor::steps(p, stride, 0), steps1 = ItemCursor::steps(p, stride, 1);
+  auto issue = [&](const ItemCursor& c, int s) {
     ptx::mbar_expect_tx(&my_bars[s], static_cast<uint32_t>(Cfg::kTileBytes));
-    ptx::tma_load_4d_hint(my_tiles + s * Cfg::kTileBytes, which ? &tmap1 : &tmap0, &my_bars[s],
-                          chunk * 64, bw * K, bh * K, b, stream_once);
+    ptx::tma_load_4d_hint(my_tiles + s * Cfg::kTileBytes, c.which ? &tmap1 : &tmap0, &my_bars[s],
+                          static_cast<int32_t>(c.chunk * 64), static_cast<int32_t>(c.bw * K),
+                          static_cast<int32_t>(c.bh * K), static_cast<int32_t>(c.b), stream_once);
   };
-  if (lane == 0) {
-    for (uint32_t i = 0; i < S && i < n_my; ++i) issue(i, i);
+  // cur: the item being transformed; ahead: the item S places further, the next to load
+  ItemCursor cur, ahead;
+  cur.decode(p, first);
+  ahead = cur;
+#pragma unroll
+  for (uint32_t i = 0; i < static_cast<uint32_t>(S); ++i) {
+    if (lane == 0 && i < n_my) issue(ahead, static_cast<int>(i));
+    ahead.advance(p, stride, ahead.which ? steps1 : steps0);
   }
 
   // A fragments of m16n8k16, row-major: a0 (row g, k 2tq..+1), a1 (row g+8, same k),
@@ -116,12 +193,9 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
     const bool ok = ptx::mbar_wait(&my_bars[s], parity, p.status, (3u << 16) | 1u);
     if (!__all_sync(0xffffffffu, ok)) break;
 
-    uint32_t item = first + idx * stride;
-    const int which = item >= p.n_items0;
-    if (which) item -= p.n_items0;
-    const uint32_t nch = static_cast<uint32_t>(p.n_chunks[which]);
-    const int blk = static_cast<int>(item / nch);
-    const int chunk = static_cast<int>(item - blk * nch);
+    const int which = static_cast<int>(cur.which);
+    const int blk = static_cast<int>(cur.blk);
+    const int chunk = static_cast<int>(cur.chunk);
     const int C = p.C[which];
     const float sc = p.scale[which];
     __nv_bfloat16* __restrict__ out = which ? out1 : out0;
@@ -153,27 +227,31 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
 
     // D fragment: d[0..1] = (row g, channels 2tq..+1), d[2..3] = (row g+8, same channels)
     const long long row0 =
-        static_cast<long long>(blk / p.bpt) * p.tile_rows + static_cast<long long>(blk % p.bpt) * p.r;
+        static_cast<long long>(cur.grp) * p.tile_rows + static_cast<long long>(cur.j) * p.r;
     const int cbase = chunk * 64 + 2 * tq;
+    // a chunk that lies inside C as a whole needs no check per group of 8 channels
+    const bool whole = chunk * 64 + 64 <= C;
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
       const int q0 = mt * 16 + g, q1 = q0 + 8;
+      __nv_bfloat16* o0 = out + (row0 + q0) * C + cbase;
+      __nv_bfloat16* o1 = o0 + 8 * static_cast<long long>(C);
+      if (q0 < p.r) {
 #pragma unroll
-      for (int nt = 0; nt < 8; ++nt) {
-        const int c = cbase + nt * 8;
-        if (c < C) {   // C is a multiple of 8: a group of 8 channels is all in or all out
-          if (q0 < p.r)
-            ptx::st_global_hint_u32(out + (row0 + q0) * C + c,
-                                    pack_bf16x2(d[mt][nt][0] * sc, d[mt][nt][1] * sc), keep);
-          if (q1 < p.r)
-            ptx::st_global_hint_u32(out + (row0 + q1) * C + c,
-                                    pack_bf16x2(d[mt][nt][2] * sc, d[mt][nt][3] * sc), keep);
-        }
+        for (int nt = 0; nt < 8; ++nt)
+          if (whole || cbase + nt * 8 < C)   // C is a multiple of 8: 8 channels are all in or all out
+            ptx::st_global_hint_u32(o0 + nt * 8, pack_bf16x2(d[mt][nt][0] * sc, d[mt][nt][1] * sc), keep);
+      }
+      if (q1 < p.r) {
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt)
+          if (whole || cbase + nt * 8 < C)
+            ptx::st_global_hint_u32(o1 + nt * 8, pack_bf16x2(d[mt][nt][2] * sc, d[mt][nt][3] * sc), keep);
       }
     }
     // rows of a padded row tile that no block owns are kept at zero
-    if ((blk % p.bpt) == p.bpt - 1 || blk == p.nb - 1) {
-      const long long tile_base = static_cast<long long>(blk / p.bpt) * p.tile_rows;
+    if (cur.j == static_cast<uint32_t>(p.bpt - 1) || blk == p.nb - 1) {
+      const long long tile_base = static_cast<long long>(cur.grp) * p.tile_rows;
       const int c = chunk * 64 + lane * 2;
       if (c < C)
         for (long long row = row0 + p.r; row < tile_base + p.tile_rows; ++row)
@@ -183,8 +261,10 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
     __syncwarp();
     if (lane == 0 && idx + S < n_my) {
       ptx::fence_proxy_async_smem();
-      issue(idx + S, s);
+      issue(ahead, s);
     }
+    ahead.advance(p, stride, ahead.which ? steps1 : steps0);
+    cur.advance(p, stride, cur.which ? steps1 : steps0);
   }
   // deferred: this grid must not complete before the kernel ahead of it has
   if (p.defer_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
