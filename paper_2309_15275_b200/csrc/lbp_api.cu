@@ -459,6 +459,17 @@ static int plan_batch(int n, const lbp_layer* layers, const lbp_basis* set, int 
         fprintf(stderr, "\n");
       }
     }
+    if (const char* e = std::getenv("LBP_BATCH_ORDER")) {   // tuning override: "1,3,2,0"
+      int o[6] = {0, 1, 2, 3, 4, 5};
+      bool seen[6] = {};
+      bool ok = std::sscanf(e, "%d,%d,%d,%d,%d,%d", &o[0], &o[1], &o[2], &o[3], &o[4], &o[5]) >= n;
+      for (int i = 0; i < n && ok; ++i) {
+        ok = o[i] >= 0 && o[i] < n && !seen[o[i]];
+        if (ok) seen[o[i]] = true;
+      }
+      if (ok)
+        for (int i = 0; i < n; ++i) best_perm[i] = o[i];
+    }
     for (int i = 0; i < n; ++i) bp.order[i] = best_perm[i];
     for (int i = 1; i < n; ++i) bp.proj_sms[i] = pps[best_perm[i - 1]][best_perm[i]];
   } else {

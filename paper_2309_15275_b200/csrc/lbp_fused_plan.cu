@@ -31,7 +31,7 @@ constexpr double kFeedBytesPerUs = 110e3;
 constexpr double kTileFixedUs = 0.3;
 // The expansion writes g_x at about 34 GB/s per SM (core butterfly); the forms
 // with extra bases or an 8 x 8 core are slower per byte.
-constexpr double kExpandBytesPerUs[3] = {34e3, 30e3, 12e3};
+constexpr double kExpandBytesPerUs[3] = {34e3, 21e3, 12e3};
 constexpr double kGwStoreBytesPerUs = 30e3;
 // K slices of g_W go through fp32 planes and one more kernel.
 constexpr double kReduceFixedUs = 3.0;

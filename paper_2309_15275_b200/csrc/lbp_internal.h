@@ -177,6 +177,8 @@ int launch_regroup_rows(const void* dense, void* grouped, int nb, int r, RowMap 
 //   LBP_BATCH_PROJ_SMS=n lbp_backward_batch: SMs given to the projection of the next
 //                        layer while the products kernel of a layer runs (0 = one
 //                        kernel at a time; unset = chosen per pair of layers)
+//   LBP_BATCH_ORDER=a,b,.. lbp_backward_batch (up to 6 problems): the order in which
+//                        the problems are taken (read at every call)
 struct TuneOptions {
   bool fused, pair, verbose, has_tiles;
   int tiles_bnw, tiles_bnx, tiles_splits;
