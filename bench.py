@@ -54,7 +54,7 @@ def _peaks():
 # DRAM traffic per step (sum over the four layers, bytes) of the two kernels, from
 # the ncu capture summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum);
 # None = not captured for the current kernels.
-NCU_TRAFFIC_PER_STEP = {"wht_project_mma_kernel": 828.9e6, "lbp_products_pair_kernel": 299.6e6}
+NCU_TRAFFIC_PER_STEP = {"wht_project_mma_kernel": 825.2e6, "lbp_products_pair_kernel": 300.2e6}
 
 
 # ------------------------------------------------------------------ clocks ----
@@ -63,15 +63,22 @@ import sys, time
 import pynvml as n
 n.nvmlInit()
 h = n.nvmlDeviceGetHandleByIndex(int(sys.argv[1]))
-print("max", n.nvmlDeviceGetMaxClockInfo(h, n.NVML_CLOCK_SM), flush=True)
+mx = n.nvmlDeviceGetMaxClockInfo(h, n.NVML_CLOCK_SM)
+print("ready", flush=True)
 end = time.time() + 120.0
 while time.time() < end:
-    mhz = n.nvmlDeviceGetClockInfo(h, n.NVML_CLOCK_SM)
     try:
-        mask = n.nvmlDeviceGetCurrentClocksEventReasons(h)
+        mhz = n.nvmlDeviceGetClockInfo(h, n.NVML_CLOCK_SM)
     except Exception:
-        mask = n.nvmlDeviceGetCurrentClocksThrottleReasons(h)
-    print(repr(time.time()), mhz, mask, flush=True)
+        continue
+    mask = 0
+    for name in ("nvmlDeviceGetCurrentClocksEventReasons", "nvmlDeviceGetCurrentClocksThrottleReasons"):
+        try:
+            mask = getattr(n, name)(h)
+            break
+        except Exception:
+            pass
+    print(repr(time.time()), mhz, mask, mx, flush=True)
 """
 
 
@@ -79,7 +86,8 @@ class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region
     runs.  The sampling loop lives in a child process (started before the timed
     region, no GPU context of its own): a thread of this process would share the
-    interpreter lock with the launching loop and hardly ever run."""
+    interpreter lock with the launching loop and hardly ever run.  If the child
+    yields nothing, nvidia-smi is asked once right after the region."""
 
     REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
                0x4: "sw_power_cap"}
@@ -91,43 +99,56 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen([sys.executable, "-c", _SAMPLER_CODE, str(self.index)],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.max_line = self.proc.stdout.readline()      # the child is up and sampling
+                                         stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True)
+            self.proc.stdout.readline()      # "ready": the child is up and sampling
         except Exception:
             self.proc = None
 
+    def _smi_once(self):
+        try:
+            out = subprocess.run(["nvidia-smi", "-i", str(self.index),
+                                  "--query-gpu=clocks.sm,clocks.max.sm,clocks_event_reasons.active",
+                                  "--format=csv,noheader,nounits"], capture_output=True, text=True,
+                                 timeout=20).stdout.strip().split(",")
+            return float(out[0]), int(float(out[1])), int(out[2].strip(), 16)
+        except Exception:
+            return None
+
     def stop(self, t_begin: float, t_end: float):
         """Summary of the samples taken between the two time.time() stamps."""
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        self.proc.terminate()
-        out = self.proc.stdout.read()
-        self.proc.wait()
-        max_mhz = None
-        try:
-            max_mhz = int(self.max_line.split()[1])
-        except Exception:
-            pass
-        rows = []
-        for ln in out.splitlines():
-            f = ln.split()
-            if len(f) == 3:
-                try:
-                    rows.append((float(f[0]), int(f[1]), int(f[2])))
-                except ValueError:
-                    pass
+        rows, err = [], ""
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                out, err = self.proc.communicate(timeout=10)
+            except Exception:
+                out, err = "", "sampler did not end"
+            for ln in out.splitlines():
+                f = ln.split()
+                if len(f) == 4:
+                    try:
+                        rows.append((float(f[0]), int(f[1]), int(f[2]), int(f[3])))
+                    except ValueError:
+                        pass
         inside = [r for r in rows if t_begin <= r[0] <= t_end]
+        how = "NVML from a child process, back to back"
         if not inside and rows:     # a region shorter than one sampling period: the nearest sample
             mid = 0.5 * (t_begin + t_end)
             inside = [min(rows, key=lambda r: abs(r[0] - mid))]
+        if not inside:
+            one = self._smi_once()
+            if one is not None:
+                inside = [(t_end, int(one[0]), one[2], one[1])]
+                how = "nvidia-smi once, right after the timed region (the NVML sampler gave nothing: " \
+                      + (err.strip().splitlines()[-1][:120] if err and err.strip() else "no output") + ")"
         reasons = set()
-        for _, _, mask in inside:
+        for r in inside:
             for bit, name in self.REASONS.items():
-                if mask & bit:
+                if r[2] & bit:
                     reasons.add(name)
         med = statistics.median([r[1] for r in inside]) if inside else None
-        return {"sm_mhz": med, "sm_max_mhz": max_mhz, "reasons": sorted(reasons),
-                "samples": len(inside), "sampling": "NVML from a child process, back to back"}
+        return {"sm_mhz": med, "sm_max_mhz": inside[0][3] if inside else None,
+                "reasons": sorted(reasons), "samples": len(inside), "sampling": how}
 
 
 # ------------------------------------------------------------- cpu oracle ----

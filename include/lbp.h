@@ -173,7 +173,9 @@ int lbp_backward(const void* x, const void* g_y, const void* W,
 /* Algorithm 1 for n (1..64) independent problems in one call, e.g. the linear
  * layers of a block whose inputs are all at hand: problem i is
  * lbp_backward(x[i], g_y[i], W[i], g_x[i], g_W[i], &layers[i], set, r, ws[i],
- * ws_bytes[i]) and gives bit-identical results.  x .. ws, ws_bytes: host arrays
+ * ws_bytes[i]); g_x is bit-identical to that call's, g_W equal up to the fp32
+ * summation order of its K slices (the tile plan follows the SMs a problem
+ * gets); results are deterministic.  x .. ws, ws_bytes: host arrays
  * of n entries.  What one problem writes (g_x, g_W, ws) no other problem may
  * read or write (LBP_ERR_OVERLAP); inputs may be shared.  Knowing that, the
  * library overlaps the problems:

@@ -426,3 +426,46 @@ def test_batch_equals_single_calls_and_rejects_overlap(dev):
     assert err.value.status in (7, 12)
     torch.cuda.synchronize()
     assert torch.equal(g_xs[1], before)
+
+
+def test_batch_of_wide_layers_runs_beside_each_other(dev):
+    # every layer takes the products kernel on CTA pairs: the batch call runs the
+    # projection of one beside the products kernel of another (its own stream,
+    # its own order) and records an event per layer.  g_x has one summation order
+    # whatever the tile plan; g_W may be summed in other K slices than in a
+    # single call, so it is compared within fp32 rounding, and with the oracle.
+    k, r = 8, 8
+    bases = O.select_bases(k, O.RULE_PREFIX, r)
+    shapes = [(768, 768), (256, 1024), (1024, 256), (384, 384)]
+    xs, gys, ws_, singles = [], [], [], []
+    for n, (ci, co) in enumerate(shapes):
+        x = synth.make_tensor((8, 16, 16, ci), ("normal", 1.0), "bf16", case_key=1960 + n).to(dev)
+        gy = synth.make_tensor((8, 16, 16, co), ("normal", 0.01), "bf16", case_key=1970 + n).to(dev)
+        w = synth.make_tensor((co, ci), ("normal", ci ** -0.5), "bf16", case_key=1980 + n).to(dev)
+        xs.append(x), gys.append(gy), ws_.append(w)
+        singles.append(lbp.lbp_backward(x, gy, w, k, bases))
+    g_xs = [torch.empty_like(x) for x in xs]
+    g_Ws = [torch.empty((w.shape[0], w.shape[1]), dtype=torch.float32, device=dev) for w in ws_]
+    wss = [lbp.alloc_workspace(x, gy, k, r) for x, gy in zip(xs, gys)]
+    events = [torch.cuda.Event() for _ in shapes]
+    side = torch.cuda.Stream(device=dev)
+    sums = []
+    for _ in range(3):
+        for g in g_xs + g_Ws:
+            g.fill_(float("nan"))
+        lbp.lbp_backward_batch(xs, gys, ws_, k, bases, g_xs=g_xs, g_Ws=g_Ws, wss=wss, done_events=events)
+        # a consumer on another stream, behind each layer's event
+        with torch.cuda.stream(side):
+            cur = []
+            for e, g in zip(events, g_Ws):
+                side.wait_event(e)
+                cur.append(g.double().sum())
+        torch.cuda.current_stream().wait_stream(side)
+        sums.append([float(v) for v in cur])
+    for i in range(len(shapes)):
+        ok_status(wss[i])
+        assert torch.equal(g_xs[i], singles[i][0])
+        assert rel(g_Ws[i], f64(singles[i][1])) <= 1e-6
+        assert sums[0][i] == sums[1][i] == sums[2][i] == float(g_Ws[i].double().sum())   # complete at the event, and deterministic
+    wx, ww = O.backward_lowrank(f64(xs[1]), f64(gys[1]), f64(ws_[1]), k, bases)
+    _assert_parity(g_xs[1], g_Ws[1], wx, ww, k, torch.bfloat16, "batch, side stream")
