@@ -195,7 +195,7 @@ static Layout plan_layout(const lbp_layer& L, int r) {
   // scratch of the persistent products kernel (bf16, r <= 16): x_hat and
   // g_y_hat with rows padded to 128-row groups
   w.fused = off = align_up(off, 1024);
-  if (r < L.k * L.k && L.dtype == LBP_BF16 && r <= 16)
+  if (r < L.k * L.k && L.dtype == LBP_BF16 && r <= fused_max_rank(L.k))
     off += fused_scratch_bytes(L, r, nullptr);
   w.total = align_up(off, 256);
   return w;
@@ -370,7 +370,7 @@ static int plan_batch(int n, const lbp_layer* layers, const lbp_basis* set, int 
     bp.proj_sms[i] = 0;
   }
   const int want = tune_options().batch_proj_sms;
-  if (n < 2 || !fused_enabled() || want == 0 || r > 16) return LBP_OK;
+  if (n < 2 || !fused_enabled() || want == 0 || r > 32) return LBP_OK;
   if (int e = check_device_arch()) return e;
   int dev = 0, sms = 0;
   LBP_CUDA_TRY(cudaGetDevice(&dev));

@@ -287,7 +287,7 @@ bool test_stall() { return g_test_stall; }
 bool fused_supported(const lbp_layer& L, const BasisPlan& bp) {
   // the epilogue addresses the tokens of a block with 32-bit element offsets
   const long long block_span = static_cast<long long>(L.k) * L.W * L.Cin;
-  return L.dtype == LBP_BF16 && (L.k == 4 || L.k == 8 || L.k == 16) && bp.r <= 16 && bp.LB <= 8 &&
+  return L.dtype == LBP_BF16 && (L.k == 4 || L.k == 8 || L.k == 16) && bp.r <= fused_max_rank(L.k) && bp.LB <= 8 &&
          bp.LB <= L.k && block_span < (1ll << 31);
 }
 

@@ -136,8 +136,8 @@ __device__ __forceinline__ void drain_tile(const FusedParams& p, const FusedBasi
     // ---- GX tile: expand g_x_hat (128 rows x BNx columns) into g_x ----
     const int m = t.group;
     const int bg = blocks_in_group(p, m);
-    // channels per thread (the 8 x 8 array of order 8 leaves registers for one)
-    constexpr int NCH = LB <= 4 ? 4 : (K >= 16 ? 2 : 1);
+    // channels per thread: an 8 x 8 coefficient array leaves registers for two
+    constexpr int NCH = LB <= 4 ? 4 : 2;
     constexpr int RUN = K / LB;
     constexpr int CPT = 32 / NCH;       // threads across one 32-column chunk
     constexpr int BSLOTS = 128 / CPT;   // blocks expanded concurrently
