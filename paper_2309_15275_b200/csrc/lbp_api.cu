@@ -370,7 +370,7 @@ static int plan_batch(int n, const lbp_layer* layers, const lbp_basis* set, int 
     bp.proj_sms[i] = 0;
   }
   const int want = tune_options().batch_proj_sms;
-  if (n < 2 || !fused_enabled() || want == 0 || r > 32) return LBP_OK;
+  if (n < 2 || !fused_enabled() || want == 0 || r > 48) return LBP_OK;
   if (int e = check_device_arch()) return e;
   int dev = 0, sms = 0;
   LBP_CUDA_TRY(cudaGetDevice(&dev));

@@ -201,52 +201,59 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
     __nv_bfloat16* __restrict__ out = which ? out1 : out0;
     const uint32_t tile = ptx::smem_u32(my_tiles + s * Cfg::kTileBytes);
 
-    float d[MT][8][4];
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-      for (int nt = 0; nt < 8; ++nt)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) d[mt][nt][j] = 0.f;
-
-#pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-      const int tok = ks * 16 + ld_tok;
-#pragma unroll
-      for (int np = 0; np < 4; ++np) {
-        const int c16 = np * 2 + ld_chunk;   // 16-byte chunk of the 128-byte token row
-        uint32_t b0, b1, b2, b3;
-        ldmatrix_x4_trans(tile + tok * 128 + ((c16 ^ (tok & 7)) << 4), b0, b1, b2, b3);
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt) {
-          mma_bf16_16816(d[mt][2 * np], afrag[mt][ks], b0, b1);
-          mma_bf16_16816(d[mt][2 * np + 1], afrag[mt][ks], b2, b3);
-        }
-      }
-    }
-
     // D fragment: d[0..1] = (row g, channels 2tq..+1), d[2..3] = (row g+8, same channels)
     const long long row0 =
         static_cast<long long>(cur.grp) * p.tile_rows + static_cast<long long>(cur.j) * p.r;
     const int cbase = chunk * 64 + 2 * tq;
     // a chunk that lies inside C as a whole needs no check per group of 8 channels
     const bool whole = chunk * 64 + 64 <= C;
+    // With three row tiles (ranks 33-48) the 64 channels are taken in two halves,
+    // so that the accumulators of a half (3 x 4 x 4 values) fit the registers.
+    constexpr int NH = MT >= 3 ? 2 : 1;
+    constexpr int NPH = 4 / NH;     // ldmatrix.x4 channel pairs per half
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-      const int q0 = mt * 16 + g, q1 = q0 + 8;
-      __nv_bfloat16* o0 = out + (row0 + q0) * C + cbase;
-      __nv_bfloat16* o1 = o0 + 8 * static_cast<long long>(C);
-      if (q0 < p.r) {
+    for (int nh = 0; nh < NH; ++nh) {
+      float d[MT][2 * NPH][4];
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt)
-          if (whole || cbase + nt * 8 < C)   // C is a multiple of 8: 8 channels are all in or all out
-            ptx::st_global_hint_u32(o0 + nt * 8, pack_bf16x2(d[mt][nt][0] * sc, d[mt][nt][1] * sc), keep);
+      for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < 2 * NPH; ++nt)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) d[mt][nt][j] = 0.f;
+
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        const int tok = ks * 16 + ld_tok;
+#pragma unroll
+        for (int npl = 0; npl < NPH; ++npl) {
+          const int c16 = (nh * NPH + npl) * 2 + ld_chunk;   // 16-byte chunk of the 128-byte token row
+          uint32_t b0, b1, b2, b3;
+          ldmatrix_x4_trans(tile + tok * 128 + ((c16 ^ (tok & 7)) << 4), b0, b1, b2, b3);
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            mma_bf16_16816(d[mt][2 * npl], afrag[mt][ks], b0, b1);
+            mma_bf16_16816(d[mt][2 * npl + 1], afrag[mt][ks], b2, b3);
+          }
+        }
       }
-      if (q1 < p.r) {
+
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt)
-          if (whole || cbase + nt * 8 < C)
-            ptx::st_global_hint_u32(o1 + nt * 8, pack_bf16x2(d[mt][nt][2] * sc, d[mt][nt][3] * sc), keep);
+      for (int mt = 0; mt < MT; ++mt) {
+        const int q0 = mt * 16 + g, q1 = q0 + 8;
+        __nv_bfloat16* o0 = out + (row0 + q0) * C + cbase + nh * (16 * NPH);
+        __nv_bfloat16* o1 = o0 + 8 * static_cast<long long>(C);
+        if (q0 < p.r) {
+#pragma unroll
+          for (int nt = 0; nt < 2 * NPH; ++nt)
+            if (whole || cbase + nh * (16 * NPH) + nt * 8 < C)   // C is a multiple of 8: 8 channels are all in or all out
+              ptx::st_global_hint_u32(o0 + nt * 8, pack_bf16x2(d[mt][nt][0] * sc, d[mt][nt][1] * sc), keep);
+        }
+        if (q1 < p.r) {
+#pragma unroll
+          for (int nt = 0; nt < 2 * NPH; ++nt)
+            if (whole || cbase + nh * (16 * NPH) + nt * 8 < C)
+              ptx::st_global_hint_u32(o1 + nt * 8, pack_bf16x2(d[mt][nt][2] * sc, d[mt][nt][3] * sc), keep);
+        }
       }
     }
     // rows of a padded row tile that no block owns are kept at zero
@@ -467,7 +474,7 @@ bool project_mma_strips(int k, int r) { return k == 4 && r <= 8; }
 
 bool project_mma_supported(int k, int r) {
   if (k == 4) return r <= 16;
-  if (k == 8) return r <= 32;
+  if (k == 8) return r <= 48;
   if (k == 16) return r <= 16;
   return false;
 }
@@ -515,7 +522,8 @@ int launch_project_mma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloa
       return launch_mma_one<4, 1>(tmaps, out0, out1, p, mp, sms, stream);
     case 8:
       if (mt == 1) return launch_mma_one<8, 1>(tmaps, out0, out1, p, mp, sms, stream);
-      return launch_mma_one<8, 2>(tmaps, out0, out1, p, mp, sms, stream);
+      if (mt == 2) return launch_mma_one<8, 2>(tmaps, out0, out1, p, mp, sms, stream);
+      return launch_mma_one<8, 3>(tmaps, out0, out1, p, mp, sms, stream);
     case 16: return launch_mma_one<16, 1>(tmaps, out0, out1, p, mp, sms, stream);
   }
   return LBP_ERR_BLOCK;
