@@ -179,7 +179,7 @@ int lbp_backward(const void* x, const void* g_y, const void* W,
  * of n entries.  What one problem writes (g_x, g_W, ws) no other problem may
  * read or write (LBP_ERR_OVERLAP); inputs may be shared.  Knowing that, the
  * library overlaps the problems:
- *  - bf16 problems of low rank (<= 16, <= 48 at k = 8) on wide layers: the projections run on a
+ *  - bf16 problems of low rank (<= 16 at k = 4, <= 48 at k = 8 and 16) on wide layers: the projections run on a
  *    stream of the library's own (one non-blocking stream and a set of events
  *    per device, created at the first such call on that device and kept: make
  *    that call outside any stream capture), the projection of one problem on

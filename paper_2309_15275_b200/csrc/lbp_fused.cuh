@@ -11,9 +11,9 @@ namespace lbp {
 
 // Highest rank the persistent products kernel takes: a 128-row group must hold
 // several blocks, and the tensor-pipe projection must produce that many rows
-// per block (order 8: up to 48, which covers LP_L1-6, LP_L1-7 and LP_L1-8 of the
-// paper's tables; orders 4 and 16: 16).
-inline int fused_max_rank(int k) { return k == 8 ? 48 : 16; }
+// per block (orders 8 and 16: up to 48, which covers LP_L1-6, LP_L1-7 and LP_L1-8
+// of the paper's tables; order 4: all 16).
+inline int fused_max_rank(int k) { return k == 4 ? 16 : 48; }
 
 // Scaling inside the products path.  Eq. 6-7 put 1/k on either side of the
 // products; all of it is powers of two, so it can sit anywhere without changing

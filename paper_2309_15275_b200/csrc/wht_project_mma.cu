@@ -167,19 +167,60 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
 
   // A fragments of m16n8k16, row-major: a0 (row g, k 2tq..+1), a1 (row g+8, same k),
   // a2 (row g, k+8), a3 (row g+8, k+8); the low half of a register is the lower k.
-  uint32_t afrag[MT][KS][4];
+  // Order 16 with more than one row tile would need 64 registers of fragments per
+  // tile.  There a k-step is one token row u of the block (16 tokens), so a
+  // fragment is its u = 0 form (which depends on v only) with the sign of
+  // wal_i(u) on top: four registers and two 16-bit sign masks per row tile.
+  constexpr bool kSignsOnTheFly = K == 16 && MT >= 2;
+  uint32_t afrag[kSignsOnTheFly ? 1 : MT][kSignsOnTheFly ? 1 : KS][4];
+  uint32_t abase[kSignsOnTheFly ? MT : 1][4];
+  uint32_t aflip[kSignsOnTheFly ? MT : 1][2];   // bit ks: wal_i(ks) = -1 for row g / g + 8
+  if constexpr (!kSignsOnTheFly) {
 #pragma unroll
-  for (int mt = 0; mt < MT; ++mt) {
+    for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
+      for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int q = mt * 16 + g + (j & 1) * 8;
+          const int tok = ks * 16 + 2 * tq + (j >> 1) * 8;
+          afrag[mt][ks][j] = basis_bits<K>(mp, q, p.r, tok) | (basis_bits<K>(mp, q, p.r, tok + 1) << 16);
+        }
+      }
+    }
+  } else {
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int q = mt * 16 + g + (j & 1) * 8;
-        const int tok = ks * 16 + 2 * tq + (j >> 1) * 8;
-        afrag[mt][ks][j] = basis_bits<K>(mp, q, p.r, tok) | (basis_bits<K>(mp, q, p.r, tok + 1) << 16);
+        const int v = 2 * tq + (j >> 1) * 8;   // token (u = 0, v)
+        abase[mt][j] = basis_bits<K>(mp, q, p.r, v) | (basis_bits<K>(mp, q, p.r, v + 1) << 16);
+      }
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int q = mt * 16 + g + h * 8;
+        uint32_t m = 0;
+        if (q < p.r)
+          for (int u = 0; u < 16; ++u) m |= static_cast<uint32_t>(__popc(mp.nat_i[q] & u) & 1) << u;
+        aflip[mt][h] = m;
       }
     }
   }
+  // fragment of row tile mt at k-step ks
+  auto a_fragment = [&](int mt, int ks, uint32_t (&a)[4]) {
+    if constexpr (!kSignsOnTheFly) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) a[j] = afrag[mt][ks][j];
+    } else {
+      const uint32_t s0 = ((aflip[mt][0] >> ks) & 1u) * 0x80008000u;
+      const uint32_t s1 = ((aflip[mt][1] >> ks) & 1u) * 0x80008000u;
+      a[0] = abase[mt][0] ^ s0;
+      a[1] = abase[mt][1] ^ s1;
+      a[2] = abase[mt][2] ^ s0;
+      a[3] = abase[mt][3] ^ s1;
+    }
+  };
 
   // ldmatrix.x4.trans source rows: lane -> matrix (lane >> 3), row (lane & 7);
   // matrices 0/1 are tokens +0..7 / +8..15 of channels 0..7 of a 16-channel pair,
@@ -211,8 +252,19 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
     // so that the accumulators of a half (3 x 4 x 4 values) fit the registers.
     constexpr int NH = MT >= 3 ? 2 : 1;
     constexpr int NPH = 4 / NH;     // ldmatrix.x4 channel pairs per half
+    // order 16 with three row tiles: 192 tensor instructions per half; unrolled
+    // as a whole the schedule runs out of registers
+    constexpr int kUnrollKs = (kSignsOnTheFly && MT >= 3) ? 4 : KS;
 #pragma unroll
     for (int nh = 0; nh < NH; ++nh) {
+      if constexpr (kSignsOnTheFly) {
+        // keep the compiler from forming all 16 fragments per row tile ahead of the
+        // loop and holding them (the register cost this form exists to avoid)
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          asm volatile("" : "+r"(aflip[mt][0]), "+r"(aflip[mt][1]));
+        }
+      }
       float d[MT][2 * NPH][4];
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt)
@@ -221,7 +273,7 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
 #pragma unroll
           for (int j = 0; j < 4; ++j) d[mt][nt][j] = 0.f;
 
-#pragma unroll
+#pragma unroll(kUnrollKs)
       for (int ks = 0; ks < KS; ++ks) {
         const int tok = ks * 16 + ld_tok;
 #pragma unroll
@@ -231,8 +283,10 @@ __global__ void __launch_bounds__(MmaCfg<K>::kWarps * 32, 1)
           ldmatrix_x4_trans(tile + tok * 128 + ((c16 ^ (tok & 7)) << 4), b0, b1, b2, b3);
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
-            mma_bf16_16816(d[mt][2 * npl], afrag[mt][ks], b0, b1);
-            mma_bf16_16816(d[mt][2 * npl + 1], afrag[mt][ks], b2, b3);
+            uint32_t a[4];
+            a_fragment(mt, ks, a);
+            mma_bf16_16816(d[mt][2 * npl], a, b0, b1);
+            mma_bf16_16816(d[mt][2 * npl + 1], a, b2, b3);
           }
         }
       }
@@ -475,7 +529,7 @@ bool project_mma_strips(int k, int r) { return k == 4 && r <= 8; }
 bool project_mma_supported(int k, int r) {
   if (k == 4) return r <= 16;
   if (k == 8) return r <= 48;
-  if (k == 16) return r <= 16;
+  if (k == 16) return r <= 48;
   return false;
 }
 
@@ -524,7 +578,10 @@ int launch_project_mma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloa
       if (mt == 1) return launch_mma_one<8, 1>(tmaps, out0, out1, p, mp, sms, stream);
       if (mt == 2) return launch_mma_one<8, 2>(tmaps, out0, out1, p, mp, sms, stream);
       return launch_mma_one<8, 3>(tmaps, out0, out1, p, mp, sms, stream);
-    case 16: return launch_mma_one<16, 1>(tmaps, out0, out1, p, mp, sms, stream);
+    case 16:
+      if (mt == 1) return launch_mma_one<16, 1>(tmaps, out0, out1, p, mp, sms, stream);
+      if (mt == 2) return launch_mma_one<16, 2>(tmaps, out0, out1, p, mp, sms, stream);
+      return launch_mma_one<16, 3>(tmaps, out0, out1, p, mp, sms, stream);
   }
   return LBP_ERR_BLOCK;
 }

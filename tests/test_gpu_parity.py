@@ -258,11 +258,11 @@ def test_bf16_full_rank_is_exact_bp(dev):
 
 # ranks chosen so that every expansion variant of the products kernel (cores of
 # 1, 2, 4 and 8 coefficients per side, the 4 x 4 core plus one or two extra
-# bases at r = 14..16, ranks up to 48 at order 8), the generic path and the full-rank mode run at
+# bases at r = 14..16, ranks up to 48 at orders 8 and 16), the generic path and the full-rank mode run at
 # full size
 @pytest.mark.parametrize("idx,ranks", [(0, (1, 2, 4, 7, 12, 16)),
                                        (1, (1, 2, 3, 5, 8, 11, 12, 13, 14, 15, 21, 28, 32, 36, 48, 50, 64)),
-                                       (2, (1, 3, 5, 10, 14, 16, 36, 100, 256))])
+                                       (2, (1, 3, 5, 10, 14, 16, 17, 21, 32, 36, 48, 49, 100, 256))])
 def test_config5_sweep_full_size(dev, idx, ranks):
     case = synth.config_cases(5)[idx]
     for r in ranks:

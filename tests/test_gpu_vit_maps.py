@@ -109,6 +109,19 @@ def test_ragged_grid_fp32_and_rectangular(dev):
         _assert_grid_parity(gx, gw, ox, ow, k, torch.float32, (k, r))
 
 
+@pytest.mark.parametrize("k,H,W,Cin,Cout,r", [(16, 20, 33, 256, 128, 6), (16, 17, 16, 64, 96, 16),
+                                               (4, 9, 6, 192, 256, 7), (8, 15, 17, 128, 384, 36),
+                                               (8, 7, 20, 64, 64, 21)])
+def test_ragged_grid_bf16_on_the_products_kernels(dev, k, H, W, Cin, Cout, r):
+    # edge blocks on both kernels of the persistent path (CTA pairs and one CTA),
+    # every order, low and high rank
+    x, gy, w = _layer(5, H, W, Cin, Cout, torch.bfloat16, 1450 + k + r)
+    bases = O.select_bases(k, O.RULE_PREFIX, r)
+    gx, gw = lbp.lbp_backward(x.to(dev), gy.to(dev), w.to(dev), k, bases)
+    ox, ow = O.backward_lowrank_padded(f64(x), f64(gy), f64(w), k, bases)
+    _assert_grid_parity(gx, gw, ox, ow, k, torch.bfloat16, (k, H, W, r))
+
+
 # ---------------- class token, bias gradient, accumulation (lbp_backward_ex) ----
 @pytest.mark.parametrize("dtype,Cin,Cout,k,bases_kind", [
     (torch.bfloat16, 384, 768, 8, "l1_4"),        # products kernel on CTA pairs, DC selected
