@@ -527,6 +527,25 @@ def _report_legs(args, torch, lbp, synth, dev, layers, k, bases, peaks, flush_bu
                           "speedup_vs_fullrank": round(full_step_us / us, 3)})
         del wss
 
+    # ---- the same step captured once and replayed as a CUDA graph ----
+    graph_row = None
+    try:
+        cap = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(cap):
+            lbp.lbp_backward_batch([L["x"] for L in layers], [L["gy"] for L in layers],
+                                   [L["w"] for L in layers], k, bases,
+                                   g_xs=[L["gx"] for L in layers], g_Ws=[L["gw"] for L in layers],
+                                   wss=[L["ws"] for L in layers])
+        us = timed(cap.replay, iters=20, warm=3)
+        roof = sum(_roof_us(peaks, L["case"].tokens, L["case"].Cin, L["case"].Cout,
+                            L["case"].blocks * RANK) for L in layers)
+        graph_row = {"us_per_step": round(us, 2), "roofline_frac": round(roof / us, 4),
+                     "tokens_per_s": tokens_per_step / (us * 1e-6)}
+        del cap
+    except Exception as exc:      # reported, never fatal: the headline is the direct call
+        graph_row = {"error": str(exc)[:200]}
+    torch.cuda.synchronize()
+
     # ---- LHE profiling pass (Sec. 3.2) on g_y of every layer ----
     lhe_rows = []
     for L in layers:
@@ -663,6 +682,7 @@ def _report_legs(args, torch, lbp, synth, dev, layers, k, bases, peaks, flush_bu
                                   "phase events, outside the timed region"},
         "layers": layer_rows,
         "rank_sweep": rank_rows,
+        "graph_replay": graph_row,
         "lhe_spectrum": lhe_rows,
         "other_configs": other,
         "gpu_launches": int(launches),

@@ -182,7 +182,9 @@ int lbp_backward(const void* x, const void* g_y, const void* W,
  *  - bf16 problems of low rank (<= 16 at k = 4, <= 48 at k = 8 and 16) on wide layers: the projections run on a
  *    stream of the library's own (one non-blocking stream and a set of events
  *    per device, created at the first such call on that device and kept: make
- *    that call outside any stream capture), the projection of one problem on
+ *    that call outside any stream capture; later calls may be captured into a
+ *    CUDA graph, the library's stream joins the capture and leaves it before
+ *    the call returns), the projection of one problem on
  *    part of the SMs beside the products kernel of another on the rest; the
  *    problems are taken in the order that leaves least of it exposed, not
  *    necessarily the given one.  Everything is ordered behind what `stream` held

@@ -469,3 +469,53 @@ def test_batch_of_wide_layers_runs_beside_each_other(dev):
         assert sums[0][i] == sums[1][i] == sums[2][i] == float(g_Ws[i].double().sum())   # complete at the event, and deterministic
     wx, ww = O.backward_lowrank(f64(xs[1]), f64(gys[1]), f64(ws_[1]), k, bases)
     _assert_parity(g_xs[1], g_Ws[1], wx, ww, k, torch.bfloat16, "batch, side stream")
+
+
+def test_batch_call_replays_from_a_cuda_graph(dev):
+    # The whole block (four layers, projections on the library's stream beside the
+    # products kernels) captured once and replayed: the replay must give what the
+    # direct call gives, also after the inputs changed in place.
+    k, r = 8, 8
+    bases = O.select_bases(k, O.RULE_PREFIX, r)
+    shapes = [(768, 768), (256, 1024), (1024, 256), (384, 384)]
+    xs, gys, ws_ = [], [], []
+    for n, (ci, co) in enumerate(shapes):
+        xs.append(synth.make_tensor((8, 16, 16, ci), ("normal", 1.0), "bf16", case_key=2060 + n).to(dev))
+        gys.append(synth.make_tensor((8, 16, 16, co), ("normal", 0.01), "bf16", case_key=2070 + n).to(dev))
+        ws_.append(synth.make_tensor((co, ci), ("normal", ci ** -0.5), "bf16", case_key=2080 + n).to(dev))
+    wss = [lbp.alloc_workspace(x, gy, k, r) for x, gy in zip(xs, gys)]
+
+    def outputs():
+        return ([torch.full_like(x, float("nan")) for x in xs],
+                [torch.full((w.shape[0], w.shape[1]), float("nan"), dtype=torch.float32, device=dev)
+                 for w in ws_])
+
+    def direct():
+        g_xs, g_Ws = outputs()
+        lbp.lbp_backward_batch(xs, gys, ws_, k, bases, g_xs=g_xs, g_Ws=g_Ws, wss=wss)
+        torch.cuda.synchronize()
+        return g_xs, g_Ws
+
+    want = direct()     # also the first call: the library makes its stream and events here
+    g_xs, g_Ws = outputs()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        lbp.lbp_backward_batch(xs, gys, ws_, k, bases, g_xs=g_xs, g_Ws=g_Ws, wss=wss)
+    for rep in range(2):
+        for g in g_xs + g_Ws:
+            g.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        for i in range(len(shapes)):
+            ok_status(wss[i])
+            assert torch.equal(g_xs[i], want[0][i]) and torch.equal(g_Ws[i], want[1][i]), (rep, i)
+    # new values in the same buffers
+    for n, x in enumerate(xs):
+        x.copy_(synth.make_tensor(tuple(x.shape), ("normal", 1.0), "bf16", case_key=2090 + n).to(dev))
+    graph.replay()
+    torch.cuda.synchronize()
+    want = direct()
+    for i in range(len(shapes)):
+        assert torch.equal(g_xs[i], want[0][i]) and torch.equal(g_Ws[i], want[1][i]), i
+    ex, ew = O.backward_lowrank(f64(xs[0]), f64(gys[0]), f64(ws_[0]), k, bases)
+    _assert_parity(g_xs[0], g_Ws[0], ex, ew, k, torch.bfloat16, "graph replay")
