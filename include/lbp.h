@@ -203,6 +203,12 @@ int lbp_backward_batch(int n, const void* const* x, const void* const* g_y, cons
                        const lbp_basis* set, int r, void* const* ws, const size_t* ws_bytes,
                        void* const* done_events, void* stream);
 
+/* Element strides of a (B,H,W,C) tensor with contiguous channels; all zero
+ * means dense (H*W*C, W*C, C). */
+typedef struct {
+  int64_t image, row, token;
+} lbp_view;
+
 /* What a linear layer of a real ViT needs around Algorithm 1 and the paper
  * leaves out (Eq. 1 has no bias; Sec. 3 knows only the tokens of the grid).
  * All pointers are device pointers; the struct itself is read on the host. */
@@ -224,6 +230,21 @@ typedef struct {
   const void* x_extra;
   const void* gy_extra;
   void* gx_extra;
+  /* Tensors that are views of larger ones (the tokens of a (B, 1 + H*W, C)
+   * sequence behind its class token; a channel slice of a wider tensor).  A
+   * view gives, in elements, the distance between consecutive images, rows and
+   * tokens of a (B,H,W,C) tensor whose C channels stay contiguous.  All three
+   * zero: dense.  Otherwise all three are positive, token >= C, and each times
+   * the element size is a multiple of 16 bytes.  The low-rank path reads and
+   * writes such tensors in place (the projection's TMA boxes and the
+   * expansion's stores take the strides); the full-rank mode (r = k*k) goes
+   * through dense copies in the workspace.  x_view is ignored when x_hat is
+   * given.  Elements of g_x between the tokens are not written. */
+  lbp_view x_view, gy_view, gx_view;
+  /* Distance in elements between consecutive extra tokens (0: dense rows);
+   * same rules as a view's strides.  With one class token per image in a
+   * (B, 1 + H*W, C) sequence this is (1 + H*W) * C. */
+  int64_t x_extra_pitch, gy_extra_pitch, gx_extra_pitch;
 } lbp_extras;
 
 /* Scratch for lbp_backward_ex (>= lbp_workspace_bytes; 0 = invalid arguments). */

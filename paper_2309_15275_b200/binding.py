@@ -41,9 +41,16 @@ class Layer(C.Structure):
                 ("dtype", C.c_int32), ("gw_dtype", C.c_int32)]
 
 
+class View(C.Structure):
+    _fields_ = [("image", C.c_int64), ("row", C.c_int64), ("token", C.c_int64)]
+
+
 class Extras(C.Structure):
     _fields_ = [("beta", C.c_float), ("g_bias", C.c_void_p), ("n_extra", C.c_int32),
-                ("x_extra", C.c_void_p), ("gy_extra", C.c_void_p), ("gx_extra", C.c_void_p)]
+                ("x_extra", C.c_void_p), ("gy_extra", C.c_void_p), ("gx_extra", C.c_void_p),
+                ("x_view", View), ("gy_view", View), ("gx_view", View),
+                ("x_extra_pitch", C.c_int64), ("gy_extra_pitch", C.c_int64),
+                ("gx_extra_pitch", C.c_int64)]
 
 
 _LIB = None
@@ -160,6 +167,33 @@ def _dev(t: torch.Tensor, name: str) -> int:
     if not t.is_contiguous():
         raise ValueError(f"{name} must be contiguous")
     return t.data_ptr()
+
+
+def _dev_view(t: torch.Tensor, name: str):
+    """Pointer and element strides of a (B,H,W,C) tensor that may be a view of a
+    larger one (channels contiguous); (0, 0, 0) stands for dense."""
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (the library has no CPU path)")
+    if t.is_contiguous():
+        return t.data_ptr(), (0, 0, 0)
+    B, H, Wd, Cc = t.shape
+    if Cc > 1 and t.stride(3) != 1:
+        raise ValueError(f"{name}: the channels of a token must be contiguous")
+    tok = t.stride(2) if Wd > 1 else Cc
+    row = t.stride(1) if H > 1 else Wd * tok
+    img = t.stride(0) if B > 1 else H * row
+    return t.data_ptr(), (img, row, tok)
+
+
+def _dev_rows(t: torch.Tensor, name: str):
+    """Pointer and row pitch (elements; 0 = dense) of an (n, C) matrix."""
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (the library has no CPU path)")
+    if t.is_contiguous():
+        return t.data_ptr(), 0
+    if t.shape[1] > 1 and t.stride(1) != 1:
+        raise ValueError(f"{name}: the channels of a token must be contiguous")
+    return t.data_ptr(), (t.stride(0) if t.shape[0] > 1 else 0)
 
 
 def _stream() -> int:
@@ -357,14 +391,18 @@ def _extras(g_y, Cin, beta, g_bias, x_extra, gy_extra, gx_extra):
             if t.dtype != g_y.dtype or t.device != g_y.device:
                 raise ValueError("extra tokens must have the layer's dtype and device")
         if n > 0:
-            ex.x_extra, ex.gy_extra, ex.gx_extra = (_dev(x_extra, "x_extra"), _dev(gy_extra, "gy_extra"),
-                                                    _dev(gx_extra, "gx_extra"))
+            ex.x_extra, ex.x_extra_pitch = _dev_rows(x_extra, "x_extra")
+            ex.gy_extra, ex.gy_extra_pitch = _dev_rows(gy_extra, "gy_extra")
+            ex.gx_extra, ex.gx_extra_pitch = _dev_rows(gx_extra, "gx_extra")
     ex.n_extra = n
     return ex
 
 
 def lbp_workspace_bytes_ex(B, H, W, Cin, Cout, k, dtype: int, gw_dtype: int, r: int, *, beta=0.0,
-                           bias=False, n_extra=0) -> int:
+                           bias=False, n_extra=0, x_view=None, gy_view=None, gx_view=None,
+                           extra_pitches=None) -> int:
+    """Scratch of lbp_backward_ex.  Views are (image, row, token) element strides,
+    extra_pitches the (x, g_y, g_x) row pitches of the extra tokens."""
     lay = _layer(B, H, W, Cin, Cout, k, dtype, gw_dtype)
     ex = Extras()
     ex.beta, ex.n_extra = float(beta), 0
@@ -372,6 +410,11 @@ def lbp_workspace_bytes_ex(B, H, W, Cin, Cout, k, dtype: int, gw_dtype: int, r: 
     ex.g_bias = 16 if bias else None
     if n_extra:
         ex.n_extra, ex.x_extra, ex.gy_extra, ex.gx_extra = int(n_extra), 16, 16, 16
+        if extra_pitches is not None:
+            ex.x_extra_pitch, ex.gy_extra_pitch, ex.gx_extra_pitch = (int(v) for v in extra_pitches)
+    for name, v in (("x_view", x_view), ("gy_view", gy_view), ("gx_view", gx_view)):
+        if v is not None:
+            setattr(ex, name, View(*[int(a) for a in v]))
     return int(_lib().lbp_workspace_bytes_ex(C.byref(lay), r, C.byref(ex)))
 
 
@@ -394,15 +437,24 @@ def lbp_backward_ex(x, g_y, W, k: int, bases, *, x_hat=None, beta: float = 0.0, 
             raise ValueError("beta != 0 accumulates into g_W: pass it")
         g_W = torch.empty((Cout, Cin), dtype=gw_dtype, device=g_y.device)
     ex = _extras(g_y, Cin, beta, g_bias, x_extra, gy_extra, gx_extra)
+    # x, g_y and g_x may be views of larger tensors (the tokens behind a class
+    # token, a channel slice): their strides go to the library as they are
+    px = None
+    if x is not None:
+        px, v = _dev_view(x, "x")
+        ex.x_view = View(*v)
+    pgy, v = _dev_view(g_y, "g_y")
+    ex.gy_view = View(*v)
+    pgx, v = _dev_view(g_x, "g_x")
+    ex.gx_view = View(*v)
     lay = _layer(B, H, Wd, Cin, Cout, k, _dtype_code(g_y.dtype), _dtype_code(g_W.dtype))
     if ws is None:
         n = int(_lib().lbp_workspace_bytes_ex(C.byref(lay), r, C.byref(ex)))
         if n == 0:
-            raise ValueError("invalid layer for lbp_workspace_bytes_ex")
+            raise ValueError("invalid layer, strides or extras for lbp_workspace_bytes_ex")
         ws = torch.empty(n, dtype=torch.uint8, device=g_y.device)
-    _check(_lib().lbp_backward_ex(None if x is None else _dev(x, "x"),
-                                  None if x_hat is None else _dev(x_hat, "x_hat"),
-                                  _dev(g_y, "g_y"), _dev(W, "W"), _dev(g_x, "g_x"), _dev(g_W, "g_W"),
+    _check(_lib().lbp_backward_ex(px, None if x_hat is None else _dev(x_hat, "x_hat"),
+                                  pgy, _dev(W, "W"), pgx, _dev(g_W, "g_W"),
                                   C.byref(lay), _bases(bases), r, C.byref(ex), _dev(ws, "ws"),
                                   ws.numel(), _stream()),
            "lbp_backward_ex")

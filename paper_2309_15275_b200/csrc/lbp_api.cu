@@ -62,19 +62,21 @@ static int get_encode_fn(EncodeTiledFn* out) {
 }
 
 int encode_block_tensor_map(CUtensorMap* map, const void* base, int dtype, int B, int H, int W,
-                            int C, int k, int box_c, bool swizzle128) {
-  return encode_box_tensor_map(map, base, dtype, B, H, W, C, box_c, k, k, swizzle128);
+                            int C, int k, int box_c, bool swizzle128, const lbp_view* view) {
+  return encode_box_tensor_map(map, base, dtype, B, H, W, C, box_c, k, k, swizzle128, view);
 }
 
 int encode_box_tensor_map(CUtensorMap* map, const void* base, int dtype, int B, int H, int W, int C,
-                          int box_c, int box_w, int box_h, bool swizzle128) {
+                          int box_c, int box_w, int box_h, bool swizzle128, const lbp_view* view) {
   EncodeTiledFn enc;
   if (int e = get_encode_fn(&enc)) return e;
   const cuuint64_t es = static_cast<cuuint64_t>(elem_size(dtype));
   const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W),
                               static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(B)};
-  const cuuint64_t strides[3] = {dims[0] * es, dims[0] * dims[1] * es,
-                                 dims[0] * dims[1] * dims[2] * es};
+  const lbp_view v = resolve_view(view, H, W, C);
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(v.token) * es,
+                                 static_cast<cuuint64_t>(v.row) * es,
+                                 static_cast<cuuint64_t>(v.image) * es};
   const cuuint32_t box[4] = {static_cast<cuuint32_t>(box_c), static_cast<cuuint32_t>(box_w),
                              static_cast<cuuint32_t>(box_h), 1u};
   const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
@@ -142,10 +144,15 @@ struct Layout {
 // tokens outside the grid) and the fp64 column-sum partials of the bias gradient.
 struct ExtrasLayout {
   size_t gw0, gw1, bias_a, bias_b, total;
+  // dense copies of tensors given as views, where a kernel wants dense operands
+  // (0: not needed): the token tensors in the full-rank mode, the extra tokens
+  size_t pack_x, pack_gy, pack_gx, ex_x, ex_gy, ex_gx;
 };
 constexpr int kBiasSlabsMax = 64;
 
-static ExtrasLayout plan_extras(const lbp_layer& L, size_t base_total) {
+static bool pitched(int64_t pitch, int C) { return pitch != 0 && pitch != C; }
+
+static ExtrasLayout plan_extras(const lbp_layer& L, size_t base_total, int r, const lbp_extras* ex) {
   ExtrasLayout e{};
   size_t off = align_up(base_total, 1024);
   const size_t gw = static_cast<size_t>(L.Cout) * L.Cin * 4;
@@ -158,6 +165,25 @@ static ExtrasLayout plan_extras(const lbp_layer& L, size_t base_total) {
   off = align_up(off + part, 1024);
   e.bias_b = off;
   off = align_up(off + part, 1024);
+  if (ex != nullptr) {
+    const size_t es = static_cast<size_t>(elem_size(L.dtype));
+    auto take = [&](size_t* where, size_t bytes) {
+      *where = off;
+      off = align_up(off + bytes, 1024);
+    };
+    if (r == L.k * L.k) {
+      const size_t T = static_cast<size_t>(L.B) * L.H * L.W;
+      if (!is_dense(&ex->x_view)) take(&e.pack_x, T * L.Cin * es);
+      if (!is_dense(&ex->gy_view)) take(&e.pack_gy, T * L.Cout * es);
+      if (!is_dense(&ex->gx_view)) take(&e.pack_gx, T * L.Cin * es);
+    }
+    if (ex->n_extra > 0) {
+      const size_t n = static_cast<size_t>(ex->n_extra);
+      if (pitched(ex->x_extra_pitch, L.Cin)) take(&e.ex_x, n * L.Cin * es);
+      if (pitched(ex->gy_extra_pitch, L.Cout)) take(&e.ex_gy, n * L.Cout * es);
+      if (pitched(ex->gx_extra_pitch, L.Cin)) take(&e.ex_gx, n * L.Cin * es);
+    }
+  }
   e.total = off;
   return e;
 }
@@ -656,15 +682,22 @@ struct CoefLoc {
 
 // Algorithm 1 after validation.  Exactly one of x / x_hat is given: x_hat are the
 // dense coefficients p(x), (blocks * r, Cin), taken earlier (Eq. 3).
+// views: strides of x, g_y, g_x when they are not dense (low-rank paths only).
 static int run_core(const void* x, const void* x_hat_in, const void* g_y, const void* W, void* g_x,
                     void* g_W, const lbp_layer& L, const BasisPlan& plan, const Layout& lay,
-                    uint8_t* wsb, cudaStream_t st, CoefLoc* gy_loc) {
+                    uint8_t* wsb, cudaStream_t st, CoefLoc* gy_loc,
+                    const CallViews* views = nullptr) {
   const int r = plan.r;
   gy_loc->ptr = nullptr;
   if (r == L.k * L.k && x_hat_in == nullptr) return run_fullrank(x, g_y, W, g_x, g_W, L, wsb, st);
 
   uint32_t* status = reinterpret_cast<uint32_t*>(wsb);
-  if (fused_enabled() && fused_supported(L, plan)) {
+  // the expansion of the products kernel addresses the tokens of an image with
+  // 32-bit offsets (dense tensors: checked by fused_supported)
+  const bool span_ok = views == nullptr || is_dense(&views->gx) ||
+                       (views->gx.row * L.H + views->gx.token * L.W < (1ll << 31) &&
+                        views->gx.image / 8 < (1ll << 31));
+  if (fused_enabled() && fused_supported(L, plan) && span_ok) {
     FusedLayout fl;
     fused_scratch_bytes(L, r, &fl);
     gy_loc->ptr = wsb + lay.fused + fl.gy_hat;
@@ -678,7 +711,7 @@ static int run_core(const void* x, const void* x_hat_in, const void* g_y, const 
       return mark_phase(2, s);
     };
     if (int e = launch_fused(x, x_hat_in, g_y, W, g_x, g_W, L, plan, wsb + lay.fused, status, st,
-                             after_projection, nullptr))
+                             after_projection, nullptr, views))
       return e;
     for (int ph = 3; ph <= 5; ++ph)
       if (int e = mark_phase(ph, st)) return e;
@@ -696,12 +729,14 @@ static int run_core(const void* x, const void* x_hat_in, const void* g_y, const 
   if (int e = mark_phase(0, st)) return e;
   if (x_hat_in != nullptr) {
     // x_hat was taken at forward time: only g_y is projected
-    if (int e = launch_project(g_y, gy_hat, L.dtype, L.B, L.H, L.W, L.Cout, plan, dense, status, st))
+    if (int e = launch_project(g_y, gy_hat, L.dtype, L.B, L.H, L.W, L.Cout, plan, dense, status, st,
+                               0.f, views ? &views->gy : nullptr))
       return e;
   } else {
     // Algorithm 1, steps 1-2: x_hat = p(x), g_y_hat = p(g_y), one launch for both
     if (int e = launch_project2(g_y, gy_hat, L.Cout, x, wsb + lay.x_hat, L.Cin, L.dtype, L.B, L.H,
-                                L.W, plan, dense, status, st))
+                                L.W, plan, dense, status, st, 0.f, 0.f, views ? &views->gy : nullptr,
+                                views ? &views->x : nullptr))
       return e;
   }
   if (int e = mark_phase(1, st)) return e;
@@ -718,22 +753,47 @@ static int run_core(const void* x, const void* x_hat_in, const void* g_y, const 
   if (int e = mark_phase(4, st)) return e;
   // step 5: g_x = p^-1(g_x_hat)
   if (int e = launch_expand(gx_hat, /*in_f32=*/true, g_x, L.dtype, L.B, L.H, L.W, L.Cin, plan,
-                            dense, st))
+                            dense, st, views ? &views->gx : nullptr))
     return e;
   return mark_phase(5, st);
 }
 
-static int check_extras(const lbp_extras* ex) {
+// A view is all zero (dense) or three positive strides, the token stride at
+// least C, each a multiple of 16 bytes and within what a tensor map can hold.
+static int check_view(const lbp_view& v, int C, int es) {
+  if (v.image == 0 && v.row == 0 && v.token == 0) return LBP_OK;
+  if (v.image <= 0 || v.row <= 0 || v.token < C) return LBP_ERR_SHAPE;
+  const int64_t lim = (int64_t{1} << 40) / es;
+  if (v.image >= lim || v.row >= lim || v.token >= lim) return LBP_ERR_SHAPE;
+  if ((v.image * es) % 16 != 0 || (v.row * es) % 16 != 0 || (v.token * es) % 16 != 0)
+    return LBP_ERR_ALIGN;
+  return LBP_OK;
+}
+
+static int check_pitch(int64_t pitch, int C, int es) {
+  if (pitch == 0) return LBP_OK;
+  if (pitch < C) return LBP_ERR_SHAPE;
+  return (pitch * es) % 16 != 0 ? LBP_ERR_ALIGN : LBP_OK;
+}
+
+static int check_extras(const lbp_extras* ex, const lbp_layer* L) {
   if (ex == nullptr) return LBP_OK;
   if (!(ex->beta == ex->beta)) return LBP_ERR_SHAPE;   // NaN
   if (ex->n_extra < 0) return LBP_ERR_SHAPE;
+  const int es = elem_size(L->dtype);
   if (ex->n_extra > 0) {
     if (ex->x_extra == nullptr || ex->gy_extra == nullptr || ex->gx_extra == nullptr)
       return LBP_ERR_NULL;
     if (!aligned16(ex->x_extra) || !aligned16(ex->gy_extra) || !aligned16(ex->gx_extra))
       return LBP_ERR_ALIGN;
+    if (int e = check_pitch(ex->x_extra_pitch, L->Cin, es)) return e;
+    if (int e = check_pitch(ex->gy_extra_pitch, L->Cout, es)) return e;
+    if (int e = check_pitch(ex->gx_extra_pitch, L->Cin, es)) return e;
   }
   if (ex->g_bias != nullptr && !aligned16(ex->g_bias)) return LBP_ERR_ALIGN;
+  if (int e = check_view(ex->x_view, L->Cin, es)) return e;
+  if (int e = check_view(ex->gy_view, L->Cout, es)) return e;
+  if (int e = check_view(ex->gx_view, L->Cin, es)) return e;
   return LBP_OK;
 }
 
@@ -742,28 +802,84 @@ static int run_backward_ex(const void* x, const void* x_hat, const void* g_y, co
                            void* g_x, void* g_W, const lbp_layer& L, const BasisPlan& plan,
                            const Layout& lay, const lbp_extras* ex, uint8_t* wsb, cudaStream_t st) {
   CoefLoc gy_loc{};
-  const bool accumulate = ex != nullptr && (ex->beta != 0.f || ex->n_extra > 0);
-  if (!accumulate && (ex == nullptr || ex->g_bias == nullptr))
+  if (ex == nullptr) return run_core(x, x_hat, g_y, W, g_x, g_W, L, plan, lay, wsb, st, &gy_loc);
+
+  CallViews cv{ex->x_view, ex->gy_view, ex->gx_view};
+  const bool strided = !is_dense(&cv.x) || !is_dense(&cv.gy) || !is_dense(&cv.gx);
+  const bool accumulate = ex->beta != 0.f || ex->n_extra > 0;
+  if (!accumulate && ex->g_bias == nullptr && !strided)
     return run_core(x, x_hat, g_y, W, g_x, g_W, L, plan, lay, wsb, st, &gy_loc);
 
-  const ExtrasLayout el = plan_extras(L, lay.total);
+  const ExtrasLayout el = plan_extras(L, lay.total, plan.r, ex);
   uint32_t* status = reinterpret_cast<uint32_t*>(wsb);
   float* gw0 = reinterpret_cast<float*>(wsb + el.gw0);
   float* gw1 = reinterpret_cast<float*>(wsb + el.gw1);
   float* sk = reinterpret_cast<float*>(wsb + lay.splitk);
+  const long long T = static_cast<long long>(L.B) * L.H * L.W;
   lbp_layer Lg = L;
   if (accumulate) Lg.gw_dtype = LBP_F32;   // this call's term in fp32, added below
-  if (int e = run_core(x, x_hat, g_y, W, g_x, accumulate ? static_cast<void*>(gw0) : g_W, Lg, plan,
-                       lay, wsb, st, &gy_loc))
-    return e;
+  void* gw_core = accumulate ? static_cast<void*>(gw0) : g_W;
+
+  // g_y as the bias gradient reads it when no coefficients serve
+  const void* gy_tokens = g_y;
+  TokenMap gy_map = token_map(resolve_view(&cv.gy, L.H, L.W, L.Cout), L.H, L.W);
+  if (plan.r == L.k * L.k && x_hat == nullptr && strided) {
+    // Eq. 2 runs on dense matrices: views go through dense copies
+    const void* xd = x;
+    const void* gyd = g_y;
+    void* gxd = g_x;
+    if (el.pack_x != 0) {
+      if (int e = launch_copy_tokens(x, wsb + el.pack_x, true, T, L.Cin, L.dtype,
+                                     token_map(cv.x, L.H, L.W), st))
+        return e;
+      xd = wsb + el.pack_x;
+    }
+    if (el.pack_gy != 0) {
+      if (int e = launch_copy_tokens(g_y, wsb + el.pack_gy, true, T, L.Cout, L.dtype,
+                                     token_map(cv.gy, L.H, L.W), st))
+        return e;
+      gyd = wsb + el.pack_gy;
+      gy_tokens = gyd;
+      gy_map = TokenMap{1, 1, L.Cout, L.Cout, L.Cout};
+    }
+    if (el.pack_gx != 0) gxd = wsb + el.pack_gx;
+    if (int e = run_core(xd, nullptr, gyd, W, gxd, gw_core, Lg, plan, lay, wsb, st, &gy_loc)) return e;
+    if (el.pack_gx != 0)
+      if (int e = launch_copy_tokens(gxd, g_x, false, T, L.Cin, L.dtype, token_map(cv.gx, L.H, L.W), st))
+        return e;
+  } else {
+    if (int e = run_core(x, x_hat, g_y, W, g_x, gw_core, Lg, plan, lay, wsb, st, &gy_loc,
+                         strided ? &cv : nullptr))
+      return e;
+  }
+  const TokenMap gye_map{1, 1, pitched(ex->gy_extra_pitch, L.Cout) ? ex->gy_extra_pitch : L.Cout, 0, 0};
   if (ex->n_extra > 0) {
-    // tokens outside the grid (a class token): Eq. 2 exactly
-    if (int e = launch_gemm(ex->gy_extra, /*a_mn_major=*/true, ex->x_extra, gw1, L.dtype, LBP_F32,
-                            L.Cout, L.Cin, ex->n_extra, sk, lay.splitk_bytes, status, st))
+    // tokens outside the grid (a class token): Eq. 2 exactly, on dense rows
+    const void* xe = ex->x_extra;
+    const void* gye = ex->gy_extra;
+    void* gxe = ex->gx_extra;
+    if (el.ex_x != 0) {
+      if (int e = launch_copy_tokens(xe, wsb + el.ex_x, true, ex->n_extra, L.Cin, L.dtype,
+                                     TokenMap{1, 1, ex->x_extra_pitch, 0, 0}, st))
+        return e;
+      xe = wsb + el.ex_x;
+    }
+    if (el.ex_gy != 0) {
+      if (int e = launch_copy_tokens(gye, wsb + el.ex_gy, true, ex->n_extra, L.Cout, L.dtype, gye_map, st))
+        return e;
+      gye = wsb + el.ex_gy;
+    }
+    if (el.ex_gx != 0) gxe = wsb + el.ex_gx;
+    if (int e = launch_gemm(gye, /*a_mn_major=*/true, xe, gw1, L.dtype, LBP_F32, L.Cout, L.Cin,
+                            ex->n_extra, sk, lay.splitk_bytes, status, st))
       return e;
-    if (int e = launch_gemm(ex->gy_extra, /*a_mn_major=*/false, W, ex->gx_extra, L.dtype, L.dtype,
-                            ex->n_extra, L.Cin, L.Cout, sk, lay.splitk_bytes, status, st))
+    if (int e = launch_gemm(gye, /*a_mn_major=*/false, W, gxe, L.dtype, L.dtype, ex->n_extra, L.Cin,
+                            L.Cout, sk, lay.splitk_bytes, status, st))
       return e;
+    if (el.ex_gx != 0)
+      if (int e = launch_copy_tokens(gxe, ex->gx_extra, false, ex->n_extra, L.Cin, L.dtype,
+                                     TokenMap{1, 1, ex->gx_extra_pitch, 0, 0}, st))
+        return e;
   }
   if (accumulate)
     if (int e = launch_gw_combine(g_W, L.gw_dtype == LBP_BF16, gw0, ex->n_extra > 0 ? gw1 : nullptr,
@@ -786,12 +902,14 @@ static int run_backward_ex(const void* x, const void* x_hat, const void* g_y, co
       if (int e = launch_column_sum(gy_loc.ptr, L.dtype, n_a, L.Cout, gy_loc.rows, plan.r, q_dc, pa, st))
         return e;
     } else {
-      n_a = static_cast<long long>(L.B) * L.H * L.W;
+      n_a = T;
       scale_a = 1.0;
-      if (int e = launch_column_sum(g_y, L.dtype, n_a, L.Cout, RowMap{1, 1}, 0, 0, pa, st)) return e;
+      if (int e = launch_column_sum(gy_tokens, L.dtype, n_a, L.Cout, RowMap{1, 1}, 0, 0, pa, st, &gy_map))
+        return e;
     }
     if (ex->n_extra > 0)
-      if (int e = launch_column_sum(ex->gy_extra, L.dtype, ex->n_extra, L.Cout, RowMap{1, 1}, 0, 0, pb, st))
+      if (int e = launch_column_sum(ex->gy_extra, L.dtype, ex->n_extra, L.Cout, RowMap{1, 1}, 0, 0, pb,
+                                    st, &gye_map))
         return e;
     if (int e = launch_bias_finish(static_cast<float*>(ex->g_bias), L.Cout, ex->beta, pa,
                                    bias_slabs(n_a), scale_a, pb, bias_slabs(ex->n_extra), st))
@@ -819,9 +937,11 @@ int lbp_backward(const void* x, const void* g_y, const void* W, void* g_x, void*
 
 size_t lbp_workspace_bytes_ex(const lbp_layer* layer, int r, const lbp_extras* ex) {
   const size_t base = lbp_workspace_bytes(layer, r);
-  if (base == 0 || check_extras(ex) != LBP_OK) return 0;
-  if (ex == nullptr || (ex->beta == 0.f && ex->n_extra == 0 && ex->g_bias == nullptr)) return base;
-  return plan_extras(*layer, base).total;
+  if (base == 0 || check_extras(ex, layer) != LBP_OK) return 0;
+  if (ex == nullptr) return base;
+  const bool strided = !is_dense(&ex->x_view) || !is_dense(&ex->gy_view) || !is_dense(&ex->gx_view);
+  if (ex->beta == 0.f && ex->n_extra == 0 && ex->g_bias == nullptr && !strided) return base;
+  return plan_extras(*layer, base, r, ex).total;
 }
 
 int lbp_backward_ex(const void* x, const void* x_hat, const void* g_y, const void* W, void* g_x,
@@ -833,7 +953,7 @@ int lbp_backward_ex(const void* x, const void* x_hat, const void* g_y, const voi
   Layout lay;
   if (int e = validate_backward(xin, g_y, W, g_x, g_W, layer, set, r, ws, ws_bytes, &plan, &lay))
     return e;
-  if (int e = check_extras(ex)) return e;
+  if (int e = check_extras(ex, layer)) return e;
   if (ws_bytes < lbp_workspace_bytes_ex(layer, r, ex)) return LBP_ERR_WORKSPACE;
   if (int e = check_device_arch()) return e;
   return run_backward_ex(x, x_hat, g_y, W, g_x, g_W, *layer, plan, lay, ex,

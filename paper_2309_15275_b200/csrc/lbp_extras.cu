@@ -57,12 +57,13 @@ __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return
 // Column sums of selected rows of a (rows, C) matrix, in fp64:
 //   partial[slab][c] = sum over the slab's rows of m[row_of(i)][c]
 // Row i of the selection is  (i / bpt) * tile_rows + (i % bpt) * r + q  (the DC
-// coefficient of block i in a projected tensor), or simply i when r == 0.
+// coefficient of block i in a projected tensor) of a dense (rows, C) matrix, or,
+// when r == 0, token i of a tensor laid out as `tm` says.
 // grid = (ceil(C / 32), slabs); block = 32 x 8: lane = channel, 8 row phases.
 template <typename T>
 __global__ void __launch_bounds__(256)
     column_sum_kernel(const T* __restrict__ m, long long n_sel, int C, int bpt, int tile_rows, int r,
-                      int q, double* __restrict__ partial) {
+                      int q, TokenMap tm, double* __restrict__ partial) {
   __shared__ double sm[8][32];
   const int lane = threadIdx.x & 31, ph = threadIdx.x >> 5;
   const int c = blockIdx.x * 32 + lane;
@@ -72,8 +73,9 @@ __global__ void __launch_bounds__(256)
   double acc = 0.0;
   if (c < C) {
     for (long long i = i0 + ph; i < i1; i += 8) {
-      const long long row = r == 0 ? i : (i / bpt) * tile_rows + (i % bpt) * r + q;
-      acc += static_cast<double>(to_f32<T>(m[row * C + c]));
+      const long long off =
+          r == 0 ? tm.offset(i) : ((i / bpt) * tile_rows + (i % bpt) * r + q) * static_cast<long long>(C);
+      acc += static_cast<double>(to_f32<T>(m[off + c]));
     }
   }
   sm[ph][lane] = acc;
@@ -132,7 +134,38 @@ __global__ void __launch_bounds__(256)
   grouped[i] = v;
 }
 
+// Moves n_tok tokens of C channels between a tensor laid out as `tm` says and a
+// dense (n_tok, C) matrix; one thread moves 16 bytes.  Strides in 16-byte units.
+__global__ void __launch_bounds__(256)
+    copy_tokens_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, long long n_vec,
+                       int row_vec, TokenMap tm16, int to_dense) {
+  const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= n_vec) return;
+  const long long tok = i / row_vec;
+  const int piece = static_cast<int>(i - tok * row_vec);
+  const long long far = tm16.offset(tok) + piece;
+  if (to_dense)
+    dst[i] = src[far];
+  else
+    dst[far] = src[i];
+}
+
 }  // namespace
+
+int launch_copy_tokens(const void* src, void* dst, bool to_dense, long long n_tok, int C, int dtype,
+                       TokenMap tm, cudaStream_t stream) {
+  if (n_tok <= 0) return LBP_OK;
+  const int es = dtype == LBP_BF16 ? 2 : 4;
+  const int per = 16 / es;   // elements per 16 bytes; every stride is a multiple of it
+  const int row_vec = C / per;
+  TokenMap tm16{tm.HW, tm.W, tm.s_image / per, tm.s_row / per, tm.s_tok / per};
+  const long long n_vec = n_tok * row_vec;
+  copy_tokens_kernel<<<static_cast<unsigned>((n_vec + 255) / 256), 256, 0, stream>>>(
+      static_cast<const uint4*>(src), static_cast<uint4*>(dst), n_vec, row_vec, tm16, to_dense ? 1 : 0);
+  count_launch();
+  LBP_CUDA_TRY(cudaGetLastError());
+  return LBP_OK;
+}
 
 int launch_gw_combine(void* g_W, bool gw_bf16, const float* a, const float* b, float beta,
                       long long mn, cudaStream_t stream) {
@@ -151,16 +184,17 @@ int bias_slabs(long long n_sel) {
 }
 
 int launch_column_sum(const void* m, int dtype, long long n_sel, int C, RowMap rows, int r, int q,
-                      double* partial, cudaStream_t stream) {
+                      double* partial, cudaStream_t stream, const TokenMap* tokens) {
+  const TokenMap tm = tokens != nullptr ? *tokens : TokenMap{1, 1, C, C, C};
   const int slabs = bias_slabs(n_sel);
   if (slabs == 0) return LBP_OK;
   dim3 grid(static_cast<unsigned>((C + 31) / 32), static_cast<unsigned>(slabs));
   if (dtype == LBP_BF16)
     column_sum_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(
-        static_cast<const __nv_bfloat16*>(m), n_sel, C, rows.bpt, rows.tile_rows, r, q, partial);
+        static_cast<const __nv_bfloat16*>(m), n_sel, C, rows.bpt, rows.tile_rows, r, q, tm, partial);
   else
     column_sum_kernel<float><<<grid, 256, 0, stream>>>(static_cast<const float*>(m), n_sel, C,
-                                                      rows.bpt, rows.tile_rows, r, q, partial);
+                                                      rows.bpt, rows.tile_rows, r, q, tm, partial);
   count_launch();
   LBP_CUDA_TRY(cudaGetLastError());
   return LBP_OK;

@@ -285,8 +285,8 @@ void set_test_stall(bool on) { g_test_stall = on; }
 bool test_stall() { return g_test_stall; }
 
 bool fused_supported(const lbp_layer& L, const BasisPlan& bp) {
-  // the epilogue addresses the tokens of a block with 32-bit element offsets
-  const long long block_span = static_cast<long long>(L.k) * L.W * L.Cin;
+  // the epilogue addresses the tokens of an image with 32-bit element offsets
+  const long long block_span = static_cast<long long>(L.H + L.k) * L.W * L.Cin;
   return L.dtype == LBP_BF16 && (L.k == 4 || L.k == 8 || L.k == 16) && bp.r <= fused_max_rank(L.k) && bp.LB <= 8 &&
          bp.LB <= L.k && block_span < (1ll << 31);
 }
@@ -380,7 +380,7 @@ int fused_project(const void* x, const void* x_hat_dense, const void* g_y, const
   int e = LBP_OK;
   if (x_hat_dense == nullptr) {
     e = launch_project2(g_y, p.gy_hat, L.Cout, x, p.x_hat, L.Cin, LBP_BF16, L.B, L.H, L.W, bp, grouped,
-                        status, ps, fused_scale_gy(L.k), fused_scale_x(L.k));
+                        status, ps, fused_scale_gy(L.k), fused_scale_x(L.k), &p.vgy, &p.vx);
   } else {
     // x_hat was taken at forward time (Eq. 3), as orthonormal coefficients: it
     // changes its row layout and its power-of-two scale
@@ -388,7 +388,7 @@ int fused_project(const void* x, const void* x_hat_dense, const void* g_y, const
                             fused_scale_x(L.k) * static_cast<float>(L.k), ps);
     if (e == LBP_OK)
       e = launch_project(g_y, p.gy_hat, LBP_BF16, L.B, L.H, L.W, L.Cout, bp, grouped, status, ps,
-                         fused_scale_gy(L.k));
+                         fused_scale_gy(L.k), &p.vgy);
   }
   if (ov != nullptr) {
     set_projection_launch(ProjLaunch{0, false, true});
@@ -401,7 +401,8 @@ int fused_project(const void* x, const void* x_hat_dense, const void* g_y, const
 
 int launch_fused(const void* x, const void* x_hat_dense, const void* g_y, const void* W, void* g_x,
                  void* g_W, const lbp_layer& L, const BasisPlan& bp, uint8_t* scratch,
-                 uint32_t* status, cudaStream_t stream, FusedPhaseHook hook, void* hook_arg) {
+                 uint32_t* status, cudaStream_t stream, FusedPhaseHook hook, void* hook_arg,
+                 const CallViews* views) {
   using namespace fused;
   FusedLayout lay;
   fused_scratch_bytes(L, bp.r, &lay);
@@ -427,6 +428,10 @@ int launch_fused(const void* x, const void* x_hat_dense, const void* g_y, const 
   p.g_x = static_cast<__nv_bfloat16*>(g_x);
   p.g_W = g_W;
   p.status = status;
+  p.vx = resolve_view(views ? &views->x : nullptr, L.H, L.W, L.Cin);
+  p.vgy = resolve_view(views ? &views->gy : nullptr, L.H, L.W, L.Cout);
+  p.vgx = resolve_view(views ? &views->gx : nullptr, L.H, L.W, L.Cin);
+  p.gx_image8 = static_cast<int32_t>(p.vgx.image / 8);
   p.test_stall = test_stall() ? 1 : 0;
   p.num_kb_x = (L.Cout + BK - 1) / BK;
   p.num_kb_w = p.G * (BM / BK);

@@ -42,6 +42,10 @@ struct FusedParams {
   __nv_bfloat16* g_x;
   void* g_W;
   uint32_t* status;
+  // element strides of x, g_y (read by the projection's tensor maps) and of g_x
+  // (the expansion's stores); dense tensors: (H*W*C, W*C, C)
+  lbp_view vx, vgy, vgx;
+  int32_t gx_image8;   // vgx.image / 8 (a multiple of 8 elements: 16 bytes of bf16)
   // failure-injection hook of the test suite (lbp_test_stall_products): the TMA
   // producers issue no load, so every other role runs into its bounded wait
   int32_t test_stall;
@@ -203,11 +207,16 @@ using FusedPhaseHook = int (*)(void* arg, cudaStream_t stream);
 
 bool fused_supported(const lbp_layer& L, const BasisPlan& bp);
 size_t fused_scratch_bytes(const lbp_layer& L, int r, FusedLayout* lay);
+// Strides of the three token tensors of a call (an entry that is all zero: dense).
+struct CallViews {
+  lbp_view x, gy, gx;
+};
 // Exactly one of x / x_hat_dense is given; x_hat_dense are coefficients p(x)
-// taken earlier, stored densely (blocks * r, Cin).
+// taken earlier, stored densely (blocks * r, Cin).  views: null = all dense.
 int launch_fused(const void* x, const void* x_hat_dense, const void* g_y, const void* W, void* g_x,
                  void* g_W, const lbp_layer& L, const BasisPlan& bp, uint8_t* scratch,
-                 uint32_t* status, cudaStream_t stream, FusedPhaseHook hook, void* hook_arg);
+                 uint32_t* status, cudaStream_t stream, FusedPhaseHook hook, void* hook_arg,
+                 const CallViews* views = nullptr);
 // Algorithm 1, steps 1-2 for the products kernel: g_y_hat (and x_hat, from x or
 // from dense coefficients) with rows padded to 128-row groups.
 int fused_project(const void* x, const void* x_hat_dense, const void* g_y, const lbp_layer& L,

@@ -143,13 +143,15 @@ __device__ __forceinline__ void drain_tile(const FusedParams& p, const FusedBasi
     constexpr int BSLOTS = 128 / CPT;   // blocks expanded concurrently
     const int cc = etid % CPT, bs = etid / CPT;
     // element offsets of a token inside a block fit 32 bits (checked on the host)
-    const int tok_stride = p.Cin, row_stride = p.W * p.Cin;
+    const int tok_stride = static_cast<int>(p.vgx.token), row_stride = static_cast<int>(p.vgx.row);
     // first token of block bl of this group (channel 0) and how many of its K x K
     // tokens lie on the grid
     auto block_origin = [&](int bl, __nv_bfloat16** o, int* ulim, int* vlim) {
       const int blk = m * p.bpt + bl;
       const int bw = blk % p.Wb, t2 = blk / p.Wb, bh = t2 % p.Hb, b = t2 / p.Hb;
-      *o = p.g_x + ((static_cast<long long>(b) * p.H + bh * K) * p.W + bw * K) * p.Cin;
+      // the offset inside one image fits 32 bits (checked on the host)
+      *o = p.g_x + (static_cast<long long>(b) * p.gx_image8 * 8 +
+                   (bh * K * row_stride + bw * K * tok_stride));
       *ulim = p.H - bh * K < K ? p.H - bh * K : K;
       *vlim = p.W - bw * K < K ? p.W - bw * K : K;
     };

@@ -73,11 +73,20 @@ void note_cuda_failure(cudaError_t e, const char* file, int line);   // LBP_VERB
 // ---- tensor maps (TMA descriptors), encoded on the host ------------------
 // 4-D channels-last tensor (B, H, W, C): box = one k x k block x box_c
 // channels; no swizzle, or the 128-byte swizzle (box_c * element size must be 128).
+// `view`: strides of a tensor that is not dense (null, or all zero: dense).
 int encode_block_tensor_map(CUtensorMap* map, const void* base, int dtype, int B, int H, int W,
-                            int C, int k, int box_c, bool swizzle128);
+                            int C, int k, int box_c, bool swizzle128,
+                            const lbp_view* view = nullptr);
 // Same tensor with an explicit box of box_h x box_w tokens.
 int encode_box_tensor_map(CUtensorMap* map, const void* base, int dtype, int B, int H, int W, int C,
-                          int box_c, int box_w, int box_h, bool swizzle128);
+                          int box_c, int box_w, int box_h, bool swizzle128,
+                          const lbp_view* view = nullptr);
+// The strides a view stands for (dense when null or all zero).
+inline lbp_view resolve_view(const lbp_view* v, int H, int W, int C) {
+  if (v != nullptr && v->token != 0) return *v;
+  return lbp_view{static_cast<int64_t>(H) * W * C, static_cast<int64_t>(W) * C, C};
+}
+inline bool is_dense(const lbp_view* v) { return v == nullptr || v->token == 0; }
 // 2-D row-major bf16 matrix (rows, cols): box = box_rows x 64 columns (128 B),
 // 128-byte swizzle.
 int encode_matrix_tensor_map(CUtensorMap* map, const void* base, long long rows, long long cols,
@@ -94,7 +103,7 @@ struct RowMap {
 // `scale` multiplies the +-1 sums; 0 selects 1/k, the orthonormal coefficients of Eq. 6.
 int launch_project(const void* t, void* t_hat, int dtype, int B, int H, int W, int C,
                    const BasisPlan& plan, RowMap rows, uint32_t* status, cudaStream_t stream,
-                   float scale = 0.f);
+                   float scale = 0.f, const lbp_view* view = nullptr);
 
 // Per-thread switch read by the projection launchers (see ProjParams::defer_wait).
 void set_projection_defer_wait(bool on);
@@ -118,7 +127,8 @@ ProjLaunch projection_launch();
 // Projects two tensors that share the token grid (x and g_y) in one launch.
 int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* out1, int C1,
                     int dtype, int B, int H, int W, const BasisPlan& plan, RowMap rows,
-                    uint32_t* status, cudaStream_t stream, float scale0 = 0.f, float scale1 = 0.f);
+                    uint32_t* status, cudaStream_t stream, float scale0 = 0.f, float scale1 = 0.f,
+                    const lbp_view* view0 = nullptr, const lbp_view* view1 = nullptr);
 
 // One-pass spectrum (bf16 data, k = 4 or 8): energy[i*k + j] of all k*k responses.
 // plan: all k*k pairs in raster order.
@@ -133,7 +143,8 @@ int launch_square_reduce(const void* t_hat, int dtype, long long rows, int C, in
 
 // t_hat is fp32 when `in_f32`, else of `dtype`; t is of `dtype`.
 int launch_expand(const void* t_hat, bool in_f32, void* t, int dtype, int B, int H, int W, int C,
-                  const BasisPlan& plan, RowMap rows, cudaStream_t stream);
+                  const BasisPlan& plan, RowMap rows, cudaStream_t stream,
+                  const lbp_view* view = nullptr);
 
 // D[M, N] = sum_k A(m, k) * B(k, n), fp32 accumulation.
 //   a_mn_major == false: A is stored (M, K) row-major;  true: A is stored (K, M) row-major.
@@ -154,12 +165,33 @@ int check_device_arch();
 // g_W <- beta * g_W + a (+ b); a, b fp32 of mn elements, g_W fp32 or bf16.
 int launch_gw_combine(void* g_W, bool gw_bf16, const float* a, const float* b, float beta,
                       long long mn, cudaStream_t stream);
-// Column sums in fp64 of n_sel selected rows of a (rows, C) matrix of `dtype`,
-// as bias_slabs(n_sel) partial rows of C doubles.  r == 0: rows 0..n_sel-1;
-// r > 0: the row of slot q of block i under the row map `rows`.
+// Where token i of a tensor of HW-token images (rows of W tokens) starts, in
+// the units of the strides: (i / HW) * s_image + ((i % HW) / W) * s_row + (i % W) * s_tok.
+// Rows with a pitch: HW = W = 1, s_image = pitch.
+struct TokenMap {
+  int32_t HW, W;
+  long long s_image, s_row, s_tok;
+  __host__ __device__ long long offset(long long i) const {
+    const long long b = i / HW;
+    const int t = static_cast<int>(i - b * HW);
+    return b * s_image + (t / W) * s_row + (t % W) * s_tok;
+  }
+};
+inline TokenMap token_map(const lbp_view& v, int H, int W) {
+  return TokenMap{H * W, W, v.image, v.row, v.token};
+}
+// Column sums in fp64 of n_sel selected rows of a matrix of `dtype`, as
+// bias_slabs(n_sel) partial rows of C doubles.  r == 0: tokens 0..n_sel-1 under
+// `tokens` (null: a dense (n_sel, C) matrix); r > 0: the row of slot q of block i
+// of a dense coefficient matrix under the row map `rows`.
 int bias_slabs(long long n_sel);
 int launch_column_sum(const void* m, int dtype, long long n_sel, int C, RowMap rows, int r, int q,
-                      double* partial, cudaStream_t stream);
+                      double* partial, cudaStream_t stream, const TokenMap* tokens = nullptr);
+// Gathers (to_dense) or scatters n_tok tokens of C channels between a tensor
+// laid out as `tm` says (element strides, multiples of 16 bytes) and a dense
+// (n_tok, C) matrix.
+int launch_copy_tokens(const void* src, void* dst, bool to_dense, long long n_tok, int C, int dtype,
+                       TokenMap tm, cudaStream_t stream);
 // g_bias[c] <- beta * g_bias[c] + scale_a * (sum of the slabs of a) + (sum of the slabs of b)
 int launch_bias_finish(float* g_bias, int C, float beta, const double* a, int slabs_a, double scale_a,
                        const double* b, int slabs_b, cudaStream_t stream);

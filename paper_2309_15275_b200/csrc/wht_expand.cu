@@ -17,6 +17,7 @@ struct ExpandParams {
   int32_t bpt, tile_rows;
   long long n_items;
   float scale;
+  long long s_image, s_row, s_tok;   // element strides of t (dense: H*W*C, W*C, C)
 };
 
 // Load the NCH channel values a lane owns from row `row` of the coefficient matrix.
@@ -68,9 +69,10 @@ __global__ void __launch_bounds__(256)
     const int bw = blk % p.Wb, bh = (blk / p.Wb) % p.Hb, b = blk / (p.Wb * p.Hb);
     const long long row0 =
         static_cast<long long>(blk / p.bpt) * p.tile_rows + static_cast<long long>(blk % p.bpt) * p.r;
-    // offset of token (u, v) of this block: tok0 + (u * W + v) * C
-    const long long tok0 =
-        ((static_cast<long long>(b) * p.H + bh * K) * p.W + bw * K) * p.C + c0;
+    // offset of token (u, v) of this block: tok0 + u * s_row + v * s_tok
+    const long long tok0 = static_cast<long long>(b) * p.s_image +
+                           static_cast<long long>(bh * K) * p.s_row +
+                           static_cast<long long>(bw * K) * p.s_tok + c0;
     // tokens of a last block that lie past the grid are not stored
     const int ulim = p.H - bh * K < K ? p.H - bh * K : K;
     const int vlim = p.W - bw * K < K ? p.W - bw * K : K;
@@ -102,7 +104,7 @@ __global__ void __launch_bounds__(256)
           for (int u = 0; u < K; ++u) {
 #pragma unroll
             for (int v = 0; v < K; ++v) {
-              store_token<TO, OUT_BF16, NCH>(t, tok0 + (static_cast<long long>(u) * p.W + v) * p.C,
+              store_token<TO, OUT_BF16, NCH>(t, tok0 + u * p.s_row + v * p.s_tok,
                                              pass, acc[u / RUN][v / RUN], p.scale);
             }
           }
@@ -112,7 +114,7 @@ __global__ void __launch_bounds__(256)
 #pragma unroll
             for (int v = 0; v < K; ++v) {
               if (u < ulim && v < vlim)
-                store_token<TO, OUT_BF16, NCH>(t, tok0 + (static_cast<long long>(u) * p.W + v) * p.C,
+                store_token<TO, OUT_BF16, NCH>(t, tok0 + u * p.s_row + v * p.s_tok,
                                                pass, acc[u / RUN][v / RUN], p.scale);
             }
           }
@@ -156,7 +158,7 @@ __global__ void __launch_bounds__(256)
               const float v1[1] = {R[vh][u]};
               if (u < ulim && vh * 4 + v_lo < vlim)
                 store_token<TO, OUT_BF16, 1>(
-                    t, tok0 + (static_cast<long long>(u) * p.W + vh * 4 + v_lo) * p.C, pass, v1,
+                    t, tok0 + u * p.s_row + (vh * 4 + v_lo) * p.s_tok, pass, v1,
                     p.scale);
             }
           }
@@ -208,9 +210,13 @@ static int launch_t(const TI* t_hat, TO* t, const ExpandParams& p, const BasisPl
 }
 
 int launch_expand(const void* t_hat, bool in_f32, void* t, int dtype, int B, int H, int W, int C,
-                  const BasisPlan& bp, RowMap rows, cudaStream_t stream) {
+                  const BasisPlan& bp, RowMap rows, cudaStream_t stream, const lbp_view* view) {
   const int K = bp.k;
   ExpandParams p;
+  const lbp_view sv = resolve_view(view, H, W, C);
+  p.s_image = sv.image;
+  p.s_row = sv.row;
+  p.s_tok = sv.token;
   p.Hb = blocks_along(H, K);
   p.Wb = blocks_along(W, K);
   p.nb = B * p.Hb * p.Wb;

@@ -255,15 +255,16 @@ static int launch_t(const CUtensorMap* tmaps, T* out0, T* out1, const ProjParams
 
 int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* out1, int C1,
                     int dtype, int B, int H, int W, const BasisPlan& bp, RowMap rows,
-                    uint32_t* status, cudaStream_t stream, float scale0, float scale1) {
+                    uint32_t* status, cudaStream_t stream, float scale0, float scale1,
+                    const lbp_view* view0, const lbp_view* view1) {
   const int K = bp.k;
   const int es = dtype == LBP_BF16 ? 2 : 4;
   const int box_c = 128 / es;   // a box wider than C is legal: the excess is zero-filled
 
   CUtensorMap tmaps[2];
-  if (int e = encode_block_tensor_map(&tmaps[0], t0, dtype, B, H, W, C0, K, box_c, false)) return e;
+  if (int e = encode_block_tensor_map(&tmaps[0], t0, dtype, B, H, W, C0, K, box_c, false, view0)) return e;
   if (t1 != nullptr) {
-    if (int e = encode_block_tensor_map(&tmaps[1], t1, dtype, B, H, W, C1, K, box_c, false)) return e;
+    if (int e = encode_block_tensor_map(&tmaps[1], t1, dtype, B, H, W, C1, K, box_c, false, view1)) return e;
   } else {
     tmaps[1] = tmaps[0];
   }
@@ -298,10 +299,10 @@ int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* ou
     CUtensorMap sw[2];
     if (project_mma_strips(K, bp.r)) {
       // order 4 works on strips of four blocks along W (4 x 16 token boxes)
-      if (int e = encode_box_tensor_map(&sw[0], t0, dtype, B, H, W, C0, box_c, 16, 4, true)) return e;
+      if (int e = encode_box_tensor_map(&sw[0], t0, dtype, B, H, W, C0, box_c, 16, 4, true, view0)) return e;
       sw[1] = sw[0];
       if (t1 != nullptr)
-        if (int e = encode_box_tensor_map(&sw[1], t1, dtype, B, H, W, C1, box_c, 16, 4, true)) return e;
+        if (int e = encode_box_tensor_map(&sw[1], t1, dtype, B, H, W, C1, box_c, 16, 4, true, view1)) return e;
       ProjParams ps = p;
       const long long strips = static_cast<long long>(B) * p.Hb * ((p.Wb + 3) / 4);
       ps.n_items0 = static_cast<uint32_t>(strips * p.n_chunks[0]);
@@ -309,10 +310,10 @@ int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* ou
       return launch_project_mma(sw, static_cast<__nv_bfloat16*>(out0),
                                 static_cast<__nv_bfloat16*>(out1), ps, bp, sms, stream);
     }
-    if (int e = encode_block_tensor_map(&sw[0], t0, dtype, B, H, W, C0, K, box_c, true)) return e;
+    if (int e = encode_block_tensor_map(&sw[0], t0, dtype, B, H, W, C0, K, box_c, true, view0)) return e;
     sw[1] = sw[0];
     if (t1 != nullptr)
-      if (int e = encode_block_tensor_map(&sw[1], t1, dtype, B, H, W, C1, K, box_c, true)) return e;
+      if (int e = encode_block_tensor_map(&sw[1], t1, dtype, B, H, W, C1, K, box_c, true, view1)) return e;
     return launch_project_mma(sw, static_cast<__nv_bfloat16*>(out0),
                               static_cast<__nv_bfloat16*>(out1), p, bp, sms, stream);
   }
@@ -329,9 +330,9 @@ int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* ou
 
 int launch_project(const void* t, void* t_hat, int dtype, int B, int H, int W, int C,
                    const BasisPlan& bp, RowMap rows, uint32_t* status, cudaStream_t stream,
-                   float scale) {
+                   float scale, const lbp_view* view) {
   return launch_project2(t, t_hat, C, nullptr, nullptr, 0, dtype, B, H, W, bp, rows, status, stream,
-                         scale, scale);
+                         scale, scale, view, nullptr);
 }
 
 }  // namespace lbp

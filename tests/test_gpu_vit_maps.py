@@ -168,6 +168,105 @@ def test_class_token_bias_and_accumulation(dev, dtype, Cin, Cout, k, bases_kind)
     assert rel(g_b, O.bias_grad(f64(gy))) <= TOL[dtype]
 
 
+# ---------------------------------------------- views of larger tensors ----
+@pytest.mark.parametrize("dtype,Cin,Cout,k,H,bases_kind", [
+    (torch.bfloat16, 192, 256, 8, 14, "l1_4"),     # products kernel on CTA pairs, ragged grid
+    (torch.bfloat16, 96, 64, 4, 7, "l1_2"),        # one-CTA products kernel
+    (torch.bfloat16, 128, 128, 8, 14, "no_dc"),    # bias read from the strided g_y
+    (torch.float32, 64, 96, 4, 7, "l1_2"),         # additions-only kernels, fp32
+    (torch.bfloat16, 128, 192, 4, 8, "full"),      # Eq. 2 through dense copies
+    (torch.float32, 64, 64, 4, 7, "full"),
+])
+def test_token_sequence_with_class_token_in_place(dev, dtype, Cin, Cout, k, H, bases_kind):
+    # A ViT sequence (B, 1 + H*W, C): the grid tokens are a view behind the class
+    # token (image stride (1 + H*W) * C), the class tokens rows with that pitch.
+    # Nothing is copied by the caller; g_x lands in the sequence's own layout.
+    B, W = 5, H
+    name = "f32" if dtype == torch.float32 else "bf16"
+    key = 2300 + Cin + k
+    xs = synth.make_tensor((B, 1 + H * W, Cin), ("normal", 1.0), name, case_key=key, tensor_id=0)
+    gys = synth.make_tensor((B, 1 + H * W, Cout), ("normal", 0.01), name, case_key=key, tensor_id=1)
+    w = synth.make_tensor((Cout, Cin), ("normal", Cin ** -0.5), name, case_key=key, tensor_id=2)
+    bases = {"l1_4": O.select_bases(k, O.RULE_L1, 4), "l1_2": O.select_bases(k, O.RULE_L1, 2),
+             "no_dc": [(0, 1), (1, 0), (1, 1)],
+             "full": O.select_bases(k, O.RULE_PREFIX, k * k)}[bases_kind]
+    xg, gyg = xs[:, 1:].reshape(B, H, W, Cin), gys[:, 1:].reshape(B, H, W, Cout)   # dense copies for the oracle
+    if bases_kind == "full":
+        ox, ow = O.backward_exact(f64(xg), f64(gyg), f64(w))
+    else:
+        ox, ow = O.backward_lowrank_padded(f64(xg), f64(gyg), f64(w), k, bases)
+    ox_cls, ow_cls = O.backward_extra_tokens(f64(xs[:, 0]), f64(gys[:, 0]), f64(w))
+    want_b = O.bias_grad(f64(gyg), f64(gys[:, 0]))
+
+    xd, gyd, wd = xs.to(dev), gys.to(dev), w.to(dev)
+    gxs = torch.full((B, 1 + H * W, Cin), float("nan"), dtype=dtype, device=dev)
+    g_b = torch.empty(Cout, dtype=torch.float32, device=dev)
+    x_view = xd[:, 1:].unflatten(1, (H, W))
+    gy_view = gyd[:, 1:].unflatten(1, (H, W))
+    gx_view = gxs[:, 1:].unflatten(1, (H, W))
+    assert not x_view.is_contiguous() and x_view.data_ptr() == xd.data_ptr() + Cin * xd.element_size()
+    _, g_W = lbp.lbp_backward_ex(x_view, gy_view, wd, k, bases, g_bias=g_b, x_extra=xd[:, 0],
+                                 gy_extra=gyd[:, 0], gx_extra=gxs[:, 0], g_x=gx_view)
+    torch.cuda.synchronize()
+    _assert_grid_parity(gxs[:, 1:].reshape(B, H, W, Cin), g_W, ox, ow + ow_cls, k, dtype, bases_kind)
+    assert rel(gxs[:, 0], ox_cls) <= TOL[dtype]
+    assert rel(g_b, want_b) <= TOL[dtype]
+    # the same call on dense copies gives the same bits
+    gx2 = torch.empty((B, H, W, Cin), dtype=dtype, device=dev)
+    gxc2 = torch.empty((B, Cin), dtype=dtype, device=dev)
+    g_b2 = torch.empty(Cout, dtype=torch.float32, device=dev)
+    _, g_W2 = lbp.lbp_backward_ex(x_view.contiguous(), gy_view.contiguous(), wd, k, bases, g_bias=g_b2,
+                                  x_extra=xd[:, 0].contiguous(), gy_extra=gyd[:, 0].contiguous(),
+                                  gx_extra=gxc2, g_x=gx2)
+    assert torch.equal(gxs[:, 1:].reshape(B, H, W, Cin), gx2) and torch.equal(gxs[:, 0], gxc2)
+    assert torch.equal(g_W, g_W2) and torch.equal(g_b, g_b2)
+
+
+@pytest.mark.parametrize("dtype,k,r", [(torch.bfloat16, 8, 8), (torch.float32, 4, 3), (torch.bfloat16, 8, 64)])
+def test_channel_slices_of_wider_tensors(dev, dtype, k, r):
+    # x, g_y and g_x are channel slices of wider tensors (token stride > C); what
+    # lies beside the slice of g_x stays untouched.
+    B, H, W, Cin, Cout = 3, 16, 24, 128, 192
+    name = "f32" if dtype == torch.float32 else "bf16"
+    x_big = synth.make_tensor((B, H, W, Cin + 64), ("normal", 1.0), name, case_key=2400 + k, tensor_id=0)
+    gy_big = synth.make_tensor((B, H, W, 2 * Cout), ("normal", 0.01), name, case_key=2400 + k, tensor_id=1)
+    w = synth.make_tensor((Cout, Cin), ("normal", Cin ** -0.5), name, case_key=2400 + k, tensor_id=2)
+    bases = O.select_bases(k, O.RULE_PREFIX, r)
+    xs, gs = x_big[..., 32:32 + Cin], gy_big[..., Cout:]
+    if r == k * k:
+        ox, ow = O.backward_exact(f64(xs), f64(gs), f64(w))
+    else:
+        ox, ow = O.backward_lowrank(f64(xs), f64(gs), f64(w), k, bases)
+    xd, gd = x_big.to(dev), gy_big.to(dev)
+    gx_big = torch.full((B, H, W, Cin + 96), 7.0, dtype=dtype, device=dev)
+    gx_view = gx_big[..., 64:64 + Cin]
+    _, g_W = lbp.lbp_backward_ex(xd[..., 32:32 + Cin], gd[..., Cout:], w.to(dev), k, bases, g_x=gx_view)
+    torch.cuda.synchronize()
+    _assert_grid_parity(gx_view.contiguous(), g_W, ox, ow, k, dtype, ("slice", r))
+    assert torch.all(gx_big[..., :64] == 7.0) and torch.all(gx_big[..., 64 + Cin:] == 7.0)
+
+
+def test_view_argument_errors(dev):
+    B, H, W, C = 2, 8, 8, 64
+    x = torch.zeros((B, H, W, C + 4), dtype=torch.bfloat16, device=dev)
+    gy = torch.zeros((B, H, W, C), dtype=torch.bfloat16, device=dev)
+    w = torch.zeros((C, C), dtype=torch.bfloat16, device=dev)
+    with pytest.raises((lbp.LbpError, ValueError)):     # token stride 68 elements: not 16-byte steps
+        lbp.lbp_backward_ex(x[..., :C], gy, w, 8, [(0, 0)])
+    with pytest.raises(ValueError):                     # channels not contiguous
+        lbp.lbp_backward_ex(torch.zeros((B, H, C, W), dtype=torch.bfloat16, device=dev).transpose(2, 3),
+                            gy, w, 8, [(0, 0)])
+    # strides in the size query: a view adds the dense copies only in the full-rank mode
+    base = lbp.lbp_workspace_bytes_ex(B, H, W, C, C, 8, lbp.LBP_BF16, lbp.LBP_F32, 8)
+    v = (H * W * 2 * C, W * 2 * C, 2 * C)
+    low = lbp.lbp_workspace_bytes_ex(B, H, W, C, C, 8, lbp.LBP_BF16, lbp.LBP_F32, 8, x_view=v)
+    full0 = lbp.lbp_workspace_bytes_ex(B, H, W, C, C, 8, lbp.LBP_BF16, lbp.LBP_F32, 64)
+    full = lbp.lbp_workspace_bytes_ex(B, H, W, C, C, 8, lbp.LBP_BF16, lbp.LBP_F32, 64, x_view=v)
+    assert low >= base and full >= full0 + B * H * W * C * 2
+    assert lbp.lbp_workspace_bytes_ex(B, H, W, C, C, 8, lbp.LBP_BF16, lbp.LBP_F32, 8,
+                                      x_view=(H * W * C, W * C, C - 8)) == 0     # token stride < C
+
+
 def test_extras_argument_errors(dev):
     x = torch.zeros((1, 8, 8, 64), dtype=torch.bfloat16, device=dev)
     gy = torch.zeros((1, 8, 8, 64), dtype=torch.bfloat16, device=dev)
@@ -240,3 +339,26 @@ def test_autograd_layer_keeps_only_the_coefficients(dev, dtype):
     assert rel(xd.grad, wx) <= TOL[dtype]
     assert rel(layer.weight.grad, ww) <= TOL[dtype]
     assert rel(layer.bias.grad, O.bias_grad(f64(gy))) <= TOL[dtype]
+
+
+@pytest.mark.parametrize("n_cls", [1, 2])
+def test_autograd_layer_on_a_token_sequence(dev, n_cls):
+    # (B, n + H*W, C) as a ViT block hands it over: the class tokens take Eq. 2,
+    # the grid tokens Algorithm 1, g_x comes back in the sequence's layout
+    k, H, W, Cin, Cout, B = 8, 14, 14, 64, 128, 3
+    dtype = torch.bfloat16
+    x = synth.make_tensor((B, n_cls + H * W, Cin), ("normal", 1.0), "bf16", case_key=1710 + n_cls)
+    gy = synth.make_tensor((B, n_cls + H * W, Cout), ("normal", 1.0), "bf16", case_key=1720 + n_cls)
+    bases = O.select_bases(k, O.RULE_L1, 4)
+    layer = lbp.LbpLinear(Cin, Cout, k, bases, device=dev, dtype=dtype, bias=True, grid=(H, W))
+    w = layer.weight.detach().clone()
+    xd = x.to(dev).requires_grad_(True)
+    layer(xd).backward(gy.to(dev))
+    xg, gyg = x[:, n_cls:].reshape(B, H, W, Cin), gy[:, n_cls:].reshape(B, H, W, Cout)
+    xc, gyc = x[:, :n_cls].reshape(B * n_cls, Cin), gy[:, :n_cls].reshape(B * n_cls, Cout)
+    wx, ww = O.backward_lowrank_padded(f64(xg), f64(gyg), f64(w), k, bases)
+    wx_cls, ww_cls = O.backward_extra_tokens(f64(xc), f64(gyc), f64(w))
+    assert rel(xd.grad[:, n_cls:].reshape(B, H, W, Cin), wx) <= TOL[dtype]
+    assert rel(xd.grad[:, :n_cls].reshape(B * n_cls, Cin), wx_cls) <= TOL[dtype]
+    assert rel(layer.weight.grad, ww + ww_cls) <= TOL[dtype]
+    assert rel(layer.bias.grad, O.bias_grad(f64(gyg), f64(gyc))) <= TOL[dtype]
