@@ -13,7 +13,7 @@ LIB = os.path.join(HERE, "liblbp.so")
 
 SOURCES = ["lbp_host.cpp", "lbp_api.cu", "wht_project.cu", "wht_project_mma.cu", "wht_expand.cu",
            "gemm_fp32.cu", "gemm_bf16.cu", "lbp_fused.cu", "lbp_fused2.cu", "lbp_static.cu",
-           "wht_spectrum.cu", "lbp_extras.cu", "lbp_fused_plan.cu"]
+           "wht_spectrum.cu", "lbp_extras.cu", "lbp_fused_plan.cu", "wht_project_umma.cu"]
 
 
 def _nvcc() -> str:

@@ -118,6 +118,8 @@ void reload_tune_options() {
   t.fused = !(e != nullptr && e[0] == '0');
   e = std::getenv("LBP_PAIR");
   t.pair = !(e != nullptr && e[0] == '0');
+  e = std::getenv("LBP_PROJECT_UMMA");
+  t.umma = !(e != nullptr && e[0] == '0');
   e = std::getenv("LBP_FUSED_VERBOSE");
   t.verbose = e != nullptr && e[0] == '1';
   e = std::getenv("LBP_FUSED_TILES");

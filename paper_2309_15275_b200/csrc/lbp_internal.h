@@ -87,6 +87,11 @@ inline lbp_view resolve_view(const lbp_view* v, int H, int W, int C) {
   return lbp_view{static_cast<int64_t>(H) * W * C, static_cast<int64_t>(W) * C, C};
 }
 inline bool is_dense(const lbp_view* v) { return v == nullptr || v->token == 0; }
+// bf16 tensor (B, H, W, C), C a multiple of 64, seen as (B, C / 64, H, W, 64):
+// box = `chunks` 64-channel chunks of one k x k block, chunk after chunk in
+// shared memory, 128-byte swizzle.
+int encode_chunked_block_tensor_map(CUtensorMap* map, const void* base, int B, int H, int W, int C,
+                                    int k, int chunks, const lbp_view* view = nullptr);
 // 2-D row-major bf16 matrix (rows, cols): box = box_rows x 64 columns (128 B),
 // 128-byte swizzle.
 int encode_matrix_tensor_map(CUtensorMap* map, const void* base, long long rows, long long cols,
@@ -204,6 +209,7 @@ int launch_regroup_rows(const void* dense, void* grouped, int nb, int r, RowMap 
 //   LBP_FUSED=0          separate product and expansion kernels instead of the
 //                        persistent products kernel
 //   LBP_PAIR=0           one-CTA products kernel also on wide layers
+//   LBP_PROJECT_UMMA=0   order-8 projection on warp-level mma.sync instead of tcgen05
 //   LBP_FUSED_TILES=a,b,c  column tiles of the two products and K slices of g_W
 //   LBP_FUSED_VERBOSE=1  print the chosen tile plan
 //   LBP_BATCH_PROJ_SMS=n lbp_backward_batch: SMs given to the projection of the next
@@ -212,7 +218,7 @@ int launch_regroup_rows(const void* dense, void* grouped, int nb, int r, RowMap 
 //   LBP_BATCH_ORDER=a,b,.. lbp_backward_batch (up to 6 problems): the order in which
 //                        the problems are taken (read at every call)
 struct TuneOptions {
-  bool fused, pair, verbose, has_tiles;
+  bool fused, pair, umma, verbose, has_tiles;
   int tiles_bnw, tiles_bnx, tiles_splits;
   int batch_proj_sms;   // -1 = library default
 };

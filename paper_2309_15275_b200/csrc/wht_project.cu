@@ -294,6 +294,21 @@ int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* ou
   LBP_CUDA_TRY(cudaGetDevice(&dev));
   LBP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
 
+  if (dtype == LBP_BF16 && tune_options().umma && project_umma_supported(K, bp.r)) {
+    // order 8 at low rank: tcgen05 kernel, an item is a block x four 64-channel chunks
+    CUtensorMap qm[2];
+    if (int e = encode_block_tensor_map(&qm[0], t0, dtype, B, H, W, C0, K, box_c, true, view0)) return e;
+    qm[1] = qm[0];
+    if (t1 != nullptr)
+      if (int e = encode_block_tensor_map(&qm[1], t1, dtype, B, H, W, C1, K, box_c, true, view1)) return e;
+    ProjParams pq = p;
+    pq.n_chunks[0] = (p.n_chunks[0] + 3) / 4;
+    pq.n_chunks[1] = t1 ? (p.n_chunks[1] + 3) / 4 : 1;
+    pq.n_items0 = static_cast<uint32_t>(static_cast<long long>(p.nb) * pq.n_chunks[0]);
+    pq.n_items = pq.n_items0 + (t1 ? static_cast<uint32_t>(static_cast<long long>(p.nb) * pq.n_chunks[1]) : 0u);
+    return launch_project_umma(qm, static_cast<__nv_bfloat16*>(out0), static_cast<__nv_bfloat16*>(out1),
+                               pq, bp, sms, stream);
+  }
   if (dtype == LBP_BF16 && project_mma_supported(K, bp.r)) {
     // bf16 data at moderate rank: the +-1 basis matrix is applied on the tensor pipe
     CUtensorMap sw[2];

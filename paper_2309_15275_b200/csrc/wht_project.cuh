@@ -40,5 +40,12 @@ bool project_mma_supported(int k, int r);
 bool project_mma_strips(int k, int r);
 int launch_project_mma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloat16* out1,
                        const ProjParams& p, const BasisPlan& bp, int sms, cudaStream_t stream);
+// Order 8, r <= 32 on the tcgen05 tensor cores (same tensor maps and parameters).
+bool project_umma_supported(int k, int r);
+int launch_project_umma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloat16* out1,
+                        const ProjParams& p, const BasisPlan& bp, int sms, cudaStream_t stream);
+// Grid size and launch attributes of a projection launch under the per-thread
+// launch shape (see ProjLaunch): `want` CTAs at most.
+int projection_grid(uint32_t want, int sms, cudaLaunchAttribute* attr, unsigned* n_attr);
 
 }  // namespace lbp

@@ -482,9 +482,7 @@ __global__ void __launch_bounds__(kStripWarps * 32, 1)
   if (p.defer_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
-// Grid size and launch attributes of a projection launch under the per-thread
-// launch shape (see ProjLaunch).
-static int projection_grid(uint32_t want, int sms, cudaLaunchAttribute* attr, unsigned* n_attr) {
+int projection_grid(uint32_t want, int sms, cudaLaunchAttribute* attr, unsigned* n_attr) {
   const ProjLaunch shape = projection_launch();
   int cap = shape.max_ctas > 0 && shape.max_ctas < sms ? shape.max_ctas : sms;
   int grid = static_cast<int>(want < static_cast<uint32_t>(cap) ? want : cap);

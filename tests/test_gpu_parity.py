@@ -204,10 +204,11 @@ def test_config3_vitb_full_size(dev, idx):
         _check_lowrank(dev, case, r)
 
 
-@pytest.mark.parametrize("switch", ["LBP_PAIR", "LBP_FUSED"])
+@pytest.mark.parametrize("switch", ["LBP_PAIR", "LBP_FUSED", "LBP_PROJECT_UMMA"])
 def test_config3_through_the_switched_paths(dev, switch):
     # LBP_PAIR=0: the one-CTA products kernel on wide layers; LBP_FUSED=0: separate
-    # product and expansion kernels.  Same bars as the default path.
+    # product and expansion kernels; LBP_PROJECT_UMMA=0: order-8 projection on warp
+    # mma.sync instead of tcgen05.  Same bars as the default path.
     os.environ[switch] = "0"
     lbp.lbp_test_reload_env()
     try:
