@@ -54,7 +54,7 @@ def _peaks():
 # DRAM traffic per step (sum over the four layers, bytes) of the two kernels, from
 # the ncu capture summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum);
 # None = not captured for the current kernels.
-NCU_TRAFFIC_PER_STEP = {"wht_project_mma_kernel": 825.2e6, "lbp_products_pair_kernel": 300.2e6}
+NCU_TRAFFIC_PER_STEP = {"wht_project_umma_kernel": 826.9e6, "lbp_products_pair_kernel": 300.5e6}
 
 
 # ------------------------------------------------------------------ clocks ----
@@ -633,9 +633,9 @@ def _report_legs(args, torch, lbp, synth, dev, layers, k, bases, peaks, flush_bu
     burst = region_s < 1.0          # short timed region at full clocks: the burst peak applies
     bf16_peak = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
     proj_ach = proj_bytes / (proj_us * 1e-6) / 1e9
-    r_proj = {"bound": "hbm", "kernel": "wht_project_mma_kernel", "achieved": round(proj_ach, 1),
+    r_proj = {"bound": "hbm", "kernel": "wht_project_umma_kernel", "achieved": round(proj_ach, 1),
               "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(proj_ach / peaks["hbm_gbs"], 4),
-              "traffic": NCU_TRAFFIC_PER_STEP["wht_project_mma_kernel"],
+              "traffic": NCU_TRAFFIC_PER_STEP["wht_project_umma_kernel"],
               "algorithmic_bytes": int(proj_bytes), "launches_per_step": len(layers),
               "us_per_step": round(proj_us, 2), "peak_source": peaks["source"],
               "share_of_step": round(proj_us / all_us, 4)}
