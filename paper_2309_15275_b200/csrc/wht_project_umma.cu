@@ -1,4 +1,4 @@
-// Projection of Eq. 6 for order 8 on the tcgen05 tensor cores (bf16, r <= 32).
+// Projection of Eq. 6 for order 8 on the tcgen05 tensor cores (bf16, r <= 48).
 //
 //   t_hat[blk, q, c] = scale * sum_tok B_q[tok] * t[blk, tok, c]
 //
@@ -20,7 +20,10 @@
 // loads at r = 16).
 //
 // Roles: warps 0-3 TMA producers (one chunk each), warp 4 MMA issuer, warps 8-11
-// and 12-15 two epilogue warpgroups (slot 0 / slot 1).  Every
+// and 12-15 two epilogue warpgroups (slot 0 / slot 1).  Ranks 33-48 (template
+// HI): the basis rows repeat every 64 rows instead of every 32, lane quarters 0
+// and 2 hold rows 0-31, quarters 1 and 3 rows 32-63; an epilogue warp then takes
+// the row half of its quarter for two of the item's chunks, one after the other.  Every
 // wait is bounded; a timeout raises the status word and all roles fall through
 // to the exit.
 #include <cuda_bf16.h>
@@ -153,11 +156,14 @@ __device__ __forceinline__ void bulk_wait_read() {
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
+template <bool HI>
 __global__ void __launch_bounds__(kThreads, 1)
     wht_project_umma_kernel(const __grid_constant__ CUtensorMap tmap0,
                             const __grid_constant__ CUtensorMap tmap1,
                             const __grid_constant__ CUtensorMap tmout0,
                             const __grid_constant__ CUtensorMap tmout1,
+                            const __grid_constant__ CUtensorMap tmout0h,   // HI: boxes of the rows from 32 on
+                            const __grid_constant__ CUtensorMap tmout1h,
                             __nv_bfloat16* __restrict__ out0, __nv_bfloat16* __restrict__ out1,
                             const __grid_constant__ ProjParams p,
                             const __grid_constant__ MmaPlan mp) {
@@ -190,11 +196,12 @@ __global__ void __launch_bounds__(kThreads, 1)
     ptx::prefetch_tensormap(&tmout0);
     ptx::prefetch_tensormap(&tmout1);
   }
-  // The basis matrix as a K-major A operand: row m holds basis m % (M / 4) (zero
-  // past r), 64 tokens = 128 bytes, 16-byte piece c of row m at piece c ^ (m & 7).
+  // The basis matrix as a K-major A operand: row m holds basis m % 32 (m % 64 at
+  // ranks above 32; zero past r), 64 tokens = 128 bytes, 16-byte piece c of row m
+  // at piece c ^ (m & 7).
   for (int e = threadIdx.x; e < M * 8; e += kThreads) {
     const int m = e >> 3, c = e & 7;
-    const int q = m % (M / 4);
+    const int q = m & (HI ? 63 : 31);
     uint32_t w[4];
 #pragma unroll
     for (int h = 0; h < 4; ++h) {
@@ -300,6 +307,10 @@ __global__ void __launch_bounds__(kThreads, 1)
     Cursor c;
     if (static_cast<uint32_t>(g) < my_quads) c.decode(p, blockIdx.x + g * gridDim.x);
     uint8_t* const my_out = smem + kOffOut + (warp - 8) * kOutBytes;
+    // rows this warp reads from its lane quarter, and the chunks it takes
+    const int half = HI ? (w & 1) : 0;
+    const int nrows = HI ? (half ? p.r - 32 : 32) : p.r;
+    constexpr int kTake = HI ? 2 : 1;
     for (uint32_t n = g; n < my_quads; n += 2) {
       const bool ok = ptx::mbar_wait(&acc_full[g], (n >> 1) & 1u, p.status, (6u << 16) | 4u);
       // one answer for the whole warp (the flag may be raised between two lanes' reads)
@@ -308,26 +319,31 @@ __global__ void __launch_bounds__(kThreads, 1)
         break;
       }
       ptx::tc_fence_after_sync();
-      uint32_t v[2][32];
-      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * w) << 16) + g * kSlotCols + w * 64;
-      ptx::tmem_ld_32x32(taddr, v[0]);
-      ptx::tmem_ld_32x32(taddr + 32, v[1]);
-      ptx::tmem_ld_wait();
-      ptx::tc_fence_before_sync();
-      if (lane == 0) ptx::mbar_arrive(&acc_empty[g]);   // the slot may be overwritten
-
       const int which = static_cast<int>(c.which);
       const int C = p.C[which];
-      const int cbase = (static_cast<int>(c.chunk) * kQuad + w) * 64;
-      if (cbase < C) {
-        const float sc = p.scale[which];
-        __nv_bfloat16* __restrict__ out = which ? out1 : out0;
-        const long long row0 =
-            static_cast<long long>(c.grp) * p.tile_rows + static_cast<long long>(c.j) * p.r;
+      const float sc = p.scale[which];
+      __nv_bfloat16* __restrict__ out = which ? out1 : out0;
+      const long long row0 =
+          static_cast<long long>(c.grp) * p.tile_rows + static_cast<long long>(c.j) * p.r;
+#pragma unroll
+      for (int ci = 0; ci < kTake; ++ci) {
+        const int cq = HI ? 2 * (w >> 1) + ci : w;   // chunk of the item
+        uint32_t v[2][32];
+        const uint32_t taddr =
+            tmem_base + (static_cast<uint32_t>(32 * w) << 16) + g * kSlotCols + cq * 64;
+        ptx::tmem_ld_32x32(taddr, v[0]);
+        ptx::tmem_ld_32x32(taddr + 32, v[1]);
+        ptx::tmem_ld_wait();
+        if (ci == kTake - 1) {
+          ptx::tc_fence_before_sync();
+          if (lane == 0) ptx::mbar_arrive(&acc_empty[g]);   // the slot may be overwritten
+        }
+        const int cbase = (static_cast<int>(c.chunk) * kQuad + cq) * 64;
+        if (cbase >= C) continue;
         // the previous store of this warp has read its rows
         if (lane == 0) bulk_wait_read();
         __syncwarp();
-        if (lane < p.r) {
+        if (lane < nrows) {
           uint8_t* orow = my_out + lane * 128;
 #pragma unroll
           for (int piece = 0; piece < 8; ++piece) {
@@ -343,11 +359,13 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
         __syncwarp();
         if (lane == 0) {
-          tma_store_2d_hint(which ? &tmout1 : &tmout0, my_out, cbase, static_cast<int32_t>(row0), keep);
+          const CUtensorMap* m = half ? (which ? &tmout1h : &tmout0h) : (which ? &tmout1 : &tmout0);
+          tma_store_2d_hint(m, my_out, cbase, static_cast<int32_t>(row0) + 32 * half, keep);
           bulk_commit();
         }
         // rows of a padded row group that no block owns are kept at zero
-        if (c.j == static_cast<uint32_t>(p.bpt - 1) || c.blk == static_cast<uint32_t>(p.nb - 1)) {
+        if (half == 0 &&
+            (c.j == static_cast<uint32_t>(p.bpt - 1) || c.blk == static_cast<uint32_t>(p.nb - 1))) {
           const long long end = static_cast<long long>(c.grp + 1) * p.tile_rows;
           const int piece = lane & 7;
           if (cbase + piece * 8 < C)   // C is a multiple of 8
@@ -372,7 +390,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 
 }  // namespace umma
 
-bool project_umma_supported(int k, int r) { return k == 8 && r <= 32; }
+bool project_umma_supported(int k, int r) { return k == 8 && r <= 48; }
 
 int launch_project_umma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloat16* out1,
                         const ProjParams& p, const BasisPlan& bp, int sms, cudaStream_t stream) {
@@ -382,15 +400,27 @@ int launch_project_umma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bflo
     mp.nat_i[q] = q < bp.r ? bp.nat_i[q] : 0;
     mp.nat_j[q] = q < bp.r ? bp.nat_j[q] : 0;
   }
-  auto kern = wht_project_umma_kernel;
-  LBP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-  // coefficient matrices as 2-D maps: a box is the r rows x 64 channels of one item
-  CUtensorMap tmout[2];
+  const bool hi = bp.r > 32;
+  auto kern = hi ? wht_project_umma_kernel<true> : wht_project_umma_kernel<false>;
+  static bool configured[2][64] = {};
+  int dev = 0;
+  LBP_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !configured[hi][dev]) {
+    LBP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    if (dev >= 0 && dev < 64) configured[hi][dev] = true;
+  }
+  // coefficient matrices as 2-D maps: a box is the rows x 64 channels of one item
+  // that one warp writes (all r rows; at ranks above 32 the first 32 and the rest)
+  CUtensorMap tmout[2], tmouth[2];
   const long long rows = (static_cast<long long>(p.nb) + p.bpt - 1) / p.bpt * p.tile_rows;
-  if (int e = encode_matrix_tensor_map(&tmout[0], out0, rows, p.C[0], bp.r)) return e;
+  if (int e = encode_matrix_tensor_map(&tmout[0], out0, rows, p.C[0], hi ? 32 : bp.r)) return e;
+  if (int e = encode_matrix_tensor_map(&tmouth[0], out0, rows, p.C[0], hi ? bp.r - 32 : bp.r)) return e;
   tmout[1] = tmout[0];
-  if (out1 != nullptr)
-    if (int e = encode_matrix_tensor_map(&tmout[1], out1, rows, p.C[1], bp.r)) return e;
+  tmouth[1] = tmouth[0];
+  if (out1 != nullptr) {
+    if (int e = encode_matrix_tensor_map(&tmout[1], out1, rows, p.C[1], hi ? 32 : bp.r)) return e;
+    if (int e = encode_matrix_tensor_map(&tmouth[1], out1, rows, p.C[1], hi ? bp.r - 32 : bp.r)) return e;
+  }
   const uint32_t want = p.n_items;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[2];
@@ -399,7 +429,8 @@ int launch_project_umma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bflo
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = stream;
   cfg.attrs = attr;
-  LBP_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmaps[0], tmaps[1], tmout[0], tmout[1], out0, out1, p, mp));
+  LBP_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmaps[0], tmaps[1], tmout[0], tmout[1], tmouth[0], tmouth[1], out0,
+                                  out1, p, mp));
   count_launch();
   LBP_CUDA_TRY(cudaGetLastError());
   return LBP_OK;
