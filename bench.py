@@ -64,6 +64,11 @@ import pynvml as n
 n.nvmlInit()
 h = n.nvmlDeviceGetHandleByIndex(int(sys.argv[1]))
 mx = n.nvmlDeviceGetMaxClockInfo(h, n.NVML_CLOCK_SM)
+for _ in range(5):          # the first queries are slow: not inside the timed region
+    try:
+        n.nvmlDeviceGetClockInfo(h, n.NVML_CLOCK_SM)
+    except Exception:
+        pass
 print("ready", flush=True)
 end = time.time() + 120.0
 while time.time() < end:
@@ -79,6 +84,7 @@ while time.time() < end:
         except Exception:
             pass
     print(repr(time.time()), mhz, mask, mx, flush=True)
+    time.sleep(0.0002)      # back-to-back NVML queries hold driver locks the launching process needs
 """
 
 
@@ -131,7 +137,7 @@ class ClockSampler:
                     except ValueError:
                         pass
         inside = [r for r in rows if t_begin <= r[0] <= t_end]
-        how = "NVML from a child process, back to back"
+        how = "NVML from a child process, every 0.2-0.3 ms"
         if not inside and rows:     # a region shorter than one sampling period: the nearest sample
             mid = 0.5 * (t_begin + t_end)
             inside = [min(rows, key=lambda r: abs(r[0] - mid))]
