@@ -21,6 +21,9 @@ extern "C" {
  * returns; the outputs of that call are undefined and the context stays
  * usable.  The paper has no counterpart; this is how the exit path behind
  * lbp_poll_status is exercised without faulting or hanging a device.
+ * `on`: bit 0 stalls the products kernels as described; bit 1 does the same to
+ * the TMA producers of the tcgen05 projection kernel (order 8, bf16, r <= 48:
+ * lbp_project and the first kernel of lbp_backward); 0 switches both off.
  * Returns LBP_OK. */
 int lbp_test_stall_products(int on);
 

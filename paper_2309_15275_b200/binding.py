@@ -581,10 +581,12 @@ def lbp_test_reload_env() -> None:
     _check(_lib().lbp_test_reload_env(), "lbp_test_reload_env")
 
 
-def lbp_test_stall_products(on: bool) -> None:
+def lbp_test_stall_products(on, projection: bool = False) -> None:
     """Test hook (include/lbp_test_hooks.h): while on, the products kernel's TMA
-    producers issue nothing, so the call ends in LBP_ERR_TIMEOUT (lbp_poll_status)."""
-    _check(_lib().lbp_test_stall_products(1 if on else 0), "lbp_test_stall_products")
+    producers (with `projection`: those of the tcgen05 projection kernel) issue
+    nothing, so the call ends in LBP_ERR_TIMEOUT (lbp_poll_status)."""
+    mode = (2 if projection else 1) if on else 0
+    _check(_lib().lbp_test_stall_products(mode), "lbp_test_stall_products")
 
 
 # ------------------------------------------------------ measurement hooks ----

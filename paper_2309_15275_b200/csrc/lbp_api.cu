@@ -599,7 +599,8 @@ int lbp_test_reload_env(void) {
 }
 
 int lbp_test_stall_products(int on) {
-  set_test_stall(on != 0);
+  set_test_stall((on & 1) != 0);
+  set_test_stall_projection((on & 2) != 0);
   return LBP_OK;
 }
 

@@ -283,6 +283,9 @@ const FusedOverlap* fused_overlap() { return g_overlap; }
 static thread_local bool g_test_stall = false;
 void set_test_stall(bool on) { g_test_stall = on; }
 bool test_stall() { return g_test_stall; }
+static thread_local bool g_test_stall_projection = false;
+void set_test_stall_projection(bool on) { g_test_stall_projection = on; }
+bool test_stall_projection() { return g_test_stall_projection; }
 
 bool fused_supported(const lbp_layer& L, const BasisPlan& bp) {
   // the epilogue addresses the tokens of an image with 32-bit element offsets

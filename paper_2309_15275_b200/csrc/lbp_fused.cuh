@@ -124,6 +124,8 @@ const FusedOverlap* fused_overlap();
 // Per-thread switch set by lbp_test_stall_products (test hook).
 void set_test_stall(bool on);
 bool test_stall();
+void set_test_stall_projection(bool on);
+bool test_stall_projection();
 
 #ifdef __CUDACC__
 // Without a table the tiles are dealt in a snake over the units (first pass

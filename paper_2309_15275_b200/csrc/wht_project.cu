@@ -7,6 +7,7 @@
 // additions only: pool to LB x LB, then a natural-order Hadamard butterfly.
 #include <cuda_bf16.h>
 
+#include "lbp_fused.cuh"
 #include "lbp_internal.h"
 #include "ptx_sm100.cuh"
 #include "wht_device.cuh"
@@ -289,6 +290,7 @@ int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* ou
   p.scale[0] = scale0 > 0.f ? scale0 : 1.0f / static_cast<float>(K);
   p.scale[1] = scale1 > 0.f ? scale1 : 1.0f / static_cast<float>(K);
   p.defer_wait = projection_defer_wait() ? 1 : 0;
+  p.test_stall = test_stall_projection() ? 1 : 0;
 
   int dev = 0, sms = 0;
   LBP_CUDA_TRY(cudaGetDevice(&dev));

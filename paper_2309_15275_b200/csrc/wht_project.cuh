@@ -24,6 +24,10 @@ struct ProjParams {
   // 1: the caller vouches that nothing this kernel touches is touched by that
   // kernel, and the wait moves to the end (it then only keeps completion ordered)
   int32_t defer_wait;
+  // failure-injection hook of the test suite (lbp_test_stall_products, bit 1):
+  // the TMA producers of the tcgen05 projection issue no load, so the other
+  // roles run into their bounded waits
+  int32_t test_stall;
 };
 
 template <int K, bool BF16>

@@ -247,7 +247,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       Cursor c;
       if (my_quads > 0) c.decode(p, blockIdx.x);
       bool ok = true;
-      for (uint32_t n = 0; n < my_quads; ++n) {
+      for (uint32_t n = 0; n < my_quads && !p.test_stall; ++n) {
         const int s = static_cast<int>(n % kStages);
         if (!ptx::mbar_wait(&empty_bar[s], ((n / kStages) + 1) & 1u, p.status, (6u << 16) | 1u)) {
           ok = false;

@@ -48,3 +48,25 @@ def test_expired_wait_is_reported_and_the_next_call_is_clean(Cin, Cout):
     assert lbp.lbp_poll_status(ws) == 0
     ox, ow = O.backward_lowrank(f64(x), f64(gy), f64(w), k, bases)
     assert O.rel_fro(f64(gx), ox) <= 2e-2 and O.rel_fro(f64(gw), ow) <= 2e-2
+
+
+def test_expired_wait_in_the_projection_kernel():
+    # the same for the tcgen05 projection kernel: no box is fetched, the tensor-core
+    # issuer and the epilogue warps give up, the status says so, the next call is clean
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    dev = torch.device("cuda:0")
+    k, r = 8, 6
+    t = synth.make_tensor((2, 16, 24, 192), ("normal", 1.0), "bf16", case_key=2500).to(dev)
+    bases = lbp.lbp_select_bases(k, lbp.SEL_PREFIX, r)
+    ws = torch.zeros(lbp.lbp_status_bytes(), dtype=torch.uint8, device=dev)
+    lbp.lbp_test_stall_products(True, projection=True)
+    try:
+        lbp.lbp_project(t, k, bases, ws=ws)
+    finally:
+        lbp.lbp_test_stall_products(False)
+    assert lbp.lbp_poll_status(ws) == LBP_ERR_TIMEOUT
+    assert lbp.lbp_poll_status(ws) == 0
+    got = lbp.lbp_project(t, k, bases, ws=ws)
+    assert lbp.lbp_poll_status(ws) == 0
+    assert O.rel_fro(f64(got), O.project(f64(t), k, bases)) <= 2e-2
