@@ -95,35 +95,6 @@ int encode_box_tensor_map(CUtensorMap* map, const void* base, int dtype, int B, 
   return LBP_OK;
 }
 
-int encode_chunked_block_tensor_map(CUtensorMap* map, const void* base, int B, int H, int W, int C,
-                                    int k, int chunks, const lbp_view* view) {
-  EncodeTiledFn enc;
-  if (int e = get_encode_fn(&enc)) return e;
-  const lbp_view v = resolve_view(view, H, W, C);
-  // (64 channels, W, H, C / 64 chunks, B): the chunk index is a dimension of its
-  // own, 128 bytes apart, so that a box lays the chunks of a block one behind
-  // the other in shared memory
-  const cuuint64_t dims[5] = {64u, static_cast<cuuint64_t>(W), static_cast<cuuint64_t>(H),
-                              static_cast<cuuint64_t>(C / 64), static_cast<cuuint64_t>(B)};
-  const cuuint64_t strides[4] = {static_cast<cuuint64_t>(v.token) * 2,
-                                 static_cast<cuuint64_t>(v.row) * 2, 128u,
-                                 static_cast<cuuint64_t>(v.image) * 2};
-  const cuuint32_t box[5] = {64u, static_cast<cuuint32_t>(k), static_cast<cuuint32_t>(k),
-                             static_cast<cuuint32_t>(chunks), 1u};
-  const cuuint32_t estr[5] = {1u, 1u, 1u, 1u, 1u};
-  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims,
-                         strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) {
-    // CUresult and cudaError_t share their numbering
-    set_last_cuda_error(static_cast<cudaError_t>(r));
-    note_cuda_failure(static_cast<cudaError_t>(r), __FILE__, __LINE__);
-    return LBP_ERR_CUDA;
-  }
-  return LBP_OK;
-}
-
 int encode_matrix_tensor_map(CUtensorMap* map, const void* base, long long rows, long long cols,
                              int box_rows) {
   EncodeTiledFn enc;

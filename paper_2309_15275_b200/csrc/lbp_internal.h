@@ -87,11 +87,6 @@ inline lbp_view resolve_view(const lbp_view* v, int H, int W, int C) {
   return lbp_view{static_cast<int64_t>(H) * W * C, static_cast<int64_t>(W) * C, C};
 }
 inline bool is_dense(const lbp_view* v) { return v == nullptr || v->token == 0; }
-// bf16 tensor (B, H, W, C), C a multiple of 64, seen as (B, C / 64, H, W, 64):
-// box = `chunks` 64-channel chunks of one k x k block, chunk after chunk in
-// shared memory, 128-byte swizzle.
-int encode_chunked_block_tensor_map(CUtensorMap* map, const void* base, int B, int H, int W, int C,
-                                    int k, int chunks, const lbp_view* view = nullptr);
 // 2-D row-major bf16 matrix (rows, cols): box = box_rows x 64 columns (128 B),
 // 128-byte swizzle.
 int encode_matrix_tensor_map(CUtensorMap* map, const void* base, long long rows, long long cols,

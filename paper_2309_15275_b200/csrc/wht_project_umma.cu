@@ -123,23 +123,6 @@ struct Cursor {
   }
 };
 
-__device__ __forceinline__ void st_global_hint_v4(void* ptr, uint4 v, uint64_t policy) {
-  asm volatile("st.global.L2::cache_hint.v4.u32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(ptr), "r"(v.x),
-               "r"(v.y), "r"(v.z), "r"(v.w), "l"(policy)
-               : "memory");
-}
-
-__device__ __forceinline__ void tma_load_5d_hint(void* smem_dst, const CUtensorMap* m, uint64_t* bar,
-                                                 int32_t c0, int32_t c1, int32_t c2, int32_t c3,
-                                                 int32_t c4, uint64_t policy) {
-  asm volatile(
-      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
-      "[%0], [%1, {%3, %4, %5, %6, %7}], [%2], %8;" ::"r"(ptx::smem_u32(smem_dst)),
-      "l"(reinterpret_cast<uint64_t>(m)), "r"(ptx::smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3),
-      "r"(c4), "l"(policy)
-      : "memory");
-}
-
 // r rows x 64 channels from shared memory (128-byte swizzle) to the coefficient matrix
 __device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap* m, const void* smem_src, int32_t x,
                                                   int32_t y, uint64_t policy) {
