@@ -296,7 +296,13 @@ int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* ou
   LBP_CUDA_TRY(cudaGetDevice(&dev));
   LBP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
 
-  if (dtype == LBP_BF16 && tune_options().umma && project_umma_supported(K, bp.r)) {
+  // The tcgen05 kernel works on four 64-channel chunks of a block at a time: with
+  // channel counts that leave many of those places empty (48 and 192 channels:
+  // half of them) the warp-level kernel is the faster one.
+  const int chunks_all = p.n_chunks[0] + (t1 ? p.n_chunks[1] : 0);
+  const int places_all = 4 * ((p.n_chunks[0] + 3) / 4 + (t1 ? (p.n_chunks[1] + 3) / 4 : 0));
+  if (dtype == LBP_BF16 && tune_options().umma && project_umma_supported(K, bp.r) &&
+      5 * chunks_all >= 4 * places_all) {
     // order 8 at low rank: tcgen05 kernel, an item is a block x four 64-channel chunks
     CUtensorMap qm[2];
     if (int e = encode_block_tensor_map(&qm[0], t0, dtype, B, H, W, C0, K, box_c, true, view0)) return e;

@@ -57,7 +57,7 @@ def test_expired_wait_in_the_projection_kernel():
         pytest.skip("no CUDA device")
     dev = torch.device("cuda:0")
     k, r = 8, 6
-    t = synth.make_tensor((2, 16, 24, 192), ("normal", 1.0), "bf16", case_key=2500).to(dev)
+    t = synth.make_tensor((2, 16, 24, 256), ("normal", 1.0), "bf16", case_key=2500).to(dev)
     bases = lbp.lbp_select_bases(k, lbp.SEL_PREFIX, r)
     ws = torch.zeros(lbp.lbp_status_bytes(), dtype=torch.uint8, device=dev)
     lbp.lbp_test_stall_products(True, projection=True)
