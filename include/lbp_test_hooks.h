@@ -22,7 +22,7 @@ extern "C" {
  * usable.  The paper has no counterpart; this is how the exit path behind
  * lbp_poll_status is exercised without faulting or hanging a device.
  * `on`: bit 0 stalls the products kernels as described; bit 1 does the same to
- * the TMA producers of the tcgen05 projection kernel (order 8, bf16, r <= 48:
+ * the TMA producers of the tcgen05 projection kernel (orders 8 and 16, bf16, r <= 48:
  * lbp_project and the first kernel of lbp_backward); 0 switches both off.
  * Returns LBP_OK. */
 int lbp_test_stall_products(int on);

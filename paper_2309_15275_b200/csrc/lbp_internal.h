@@ -204,7 +204,7 @@ int launch_regroup_rows(const void* dense, void* grouped, int nb, int r, RowMap 
 //   LBP_FUSED=0          separate product and expansion kernels instead of the
 //                        persistent products kernel
 //   LBP_PAIR=0           one-CTA products kernel also on wide layers
-//   LBP_PROJECT_UMMA=0   order-8 projection on warp-level mma.sync instead of tcgen05
+//   LBP_PROJECT_UMMA=0   projection of orders 8 and 16 on warp-level mma.sync instead of tcgen05
 //   LBP_FUSED_TILES=a,b,c  column tiles of the two products and K slices of g_W
 //   LBP_FUSED_VERBOSE=1  print the chosen tile plan
 //   LBP_BATCH_PROJ_SMS=n lbp_backward_batch: SMs given to the projection of the next

@@ -303,12 +303,14 @@ int launch_project2(const void* t0, void* out0, int C0, const void* t1, void* ou
   const int places_all = 4 * ((p.n_chunks[0] + 3) / 4 + (t1 ? (p.n_chunks[1] + 3) / 4 : 0));
   if (dtype == LBP_BF16 && tune_options().umma && project_umma_supported(K, bp.r) &&
       5 * chunks_all >= 4 * places_all) {
-    // order 8 at low rank: tcgen05 kernel, an item is a block x four 64-channel chunks
+    // orders 8 and 16 at low rank: tcgen05 kernel, an item is a block x four 64-channel chunks
     CUtensorMap qm[2];
-    if (int e = encode_block_tensor_map(&qm[0], t0, dtype, B, H, W, C0, K, box_c, true, view0)) return e;
+    // a box is 64 tokens: the block at order 8, four of its token rows at order 16
+    const int box_h = 64 / K;
+    if (int e = encode_box_tensor_map(&qm[0], t0, dtype, B, H, W, C0, box_c, K, box_h, true, view0)) return e;
     qm[1] = qm[0];
     if (t1 != nullptr)
-      if (int e = encode_block_tensor_map(&qm[1], t1, dtype, B, H, W, C1, K, box_c, true, view1)) return e;
+      if (int e = encode_box_tensor_map(&qm[1], t1, dtype, B, H, W, C1, box_c, K, box_h, true, view1)) return e;
     ProjParams pq = p;
     pq.n_chunks[0] = (p.n_chunks[0] + 3) / 4;
     pq.n_chunks[1] = t1 ? (p.n_chunks[1] + 3) / 4 : 1;

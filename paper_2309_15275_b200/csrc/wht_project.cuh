@@ -44,7 +44,8 @@ bool project_mma_supported(int k, int r);
 bool project_mma_strips(int k, int r);
 int launch_project_mma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloat16* out1,
                        const ProjParams& p, const BasisPlan& bp, int sms, cudaStream_t stream);
-// Order 8, r <= 32 on the tcgen05 tensor cores (same tensor maps and parameters).
+// Orders 8 and 16, r <= 48 on the tcgen05 tensor cores (boxes of 64 tokens; in the
+// parameters n_chunks counts items of four 64-channel chunks per block).
 bool project_umma_supported(int k, int r);
 int launch_project_umma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloat16* out1,
                         const ProjParams& p, const BasisPlan& bp, int sms, cudaStream_t stream);

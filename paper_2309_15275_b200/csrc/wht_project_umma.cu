@@ -1,4 +1,4 @@
-// Projection of Eq. 6 for order 8 on the tcgen05 tensor cores (bf16, r <= 48).
+// Projection of Eq. 6 for orders 8 and 16 on the tcgen05 tensor cores (bf16, r <= 48).
 //
 //   t_hat[blk, q, c] = scale * sum_tok B_q[tok] * t[blk, tok, c]
 //
@@ -19,6 +19,11 @@
 // (per-lane stores of 16 bytes to r different rows cost the SM more than the
 // loads at r = 16).
 //
+// Order 16 (template K): a block's 256 tokens are taken as four parts of 64
+// (four token rows each, a 4 x 16 box), every part a stage of its own with its
+// own 64 columns of the basis matrix, and the four parts accumulate in the same
+// accumulator slot: the tile, stage and epilogue shapes stay those of order 8.
+//
 // Roles: warps 0-3 TMA producers (one chunk each), warp 4 MMA issuer, warps 8-11
 // and 12-15 two epilogue warpgroups (slot 0 / slot 1).  Ranks 33-48 (template
 // HI): the basis rows repeat every 64 rows instead of every 32, lane quarters 0
@@ -37,21 +42,25 @@
 namespace lbp {
 namespace umma {
 
-constexpr int K = 8;
-constexpr int kTileBytes = K * K * 128;          // 64 tokens x 64 channels of bf16
+constexpr int kTileBytes = 64 * 128;             // 64 tokens x 64 channels of bf16
 constexpr int M = 128;                           // rows of the tensor-core tile
 constexpr int kQuad = 4;                         // 64-channel chunks per item = per stage = per accumulator slot
 constexpr int kStageBytes = kQuad * kTileBytes;  // 32 KB
-constexpr int kStages = 5;
 constexpr int kProducers = 4;                    // warps 0-3: each fetches one chunk of an item
-constexpr int kABytes = 128 * 128;               // basis matrix: 128 rows x 64 tokens of bf16
+constexpr int kPanelBytes = 128 * 128;           // basis matrix for 64 tokens: 128 rows x 128 bytes
 constexpr int kOutBytes = 32 * 128;              // an epilogue warp's rows on their way out
 constexpr int kThreads = 16 * 32;
-constexpr int kOffA = kStages * kStageBytes;
-constexpr int kOffOut = kOffA + kABytes;
-constexpr int kOffBar = kOffOut + 8 * kOutBytes;
-constexpr int kSmemBytes = kOffBar + 256 + 1024;
-static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA exceeded");
+// Per order: parts of 64 tokens per block, stages of the ring, shared-memory map.
+template <int K>
+struct Cfg {
+  static constexpr int kParts = K * K / 64;
+  static constexpr int kStages = K == 8 ? 5 : 4;
+  static constexpr int kOffA = kStages * kStageBytes;
+  static constexpr int kOffOut = kOffA + kParts * kPanelBytes;
+  static constexpr int kOffBar = kOffOut + 8 * kOutBytes;
+  static constexpr int kSmemBytes = kOffBar + 256 + 1024;
+  static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA exceeded");
+};
 constexpr uint32_t kTmemCols = 512, kSlotCols = 256;
 
 // One item (block x four 64-channel chunks of one of the two tensors; in
@@ -139,7 +148,7 @@ __device__ __forceinline__ void bulk_wait_read() {
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
-template <bool HI>
+template <int K, bool HI>
 __global__ void __launch_bounds__(kThreads, 1)
     wht_project_umma_kernel(const __grid_constant__ CUtensorMap tmap0,
                             const __grid_constant__ CUtensorMap tmap1,
@@ -153,8 +162,9 @@ __global__ void __launch_bounds__(kThreads, 1)
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-  uint8_t* sA = smem + kOffA;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kOffBar);
+  constexpr int kStages = Cfg<K>::kStages, kParts = Cfg<K>::kParts;
+  uint8_t* sA = smem + Cfg<K>::kOffA;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg<K>::kOffBar);
   uint64_t* empty_bar = full_bar + kStages;
   uint64_t* acc_full = empty_bar + kStages;   // [2]
   uint64_t* acc_empty = acc_full + 2;         // [2]
@@ -179,19 +189,20 @@ __global__ void __launch_bounds__(kThreads, 1)
     ptx::prefetch_tensormap(&tmout0);
     ptx::prefetch_tensormap(&tmout1);
   }
-  // The basis matrix as a K-major A operand: row m holds basis m % 32 (m % 64 at
-  // ranks above 32; zero past r), 64 tokens = 128 bytes, 16-byte piece c of row m
-  // at piece c ^ (m & 7).
-  for (int e = threadIdx.x; e < M * 8; e += kThreads) {
-    const int m = e >> 3, c = e & 7;
+  // The basis matrix as K-major A operands, one panel per part of 64 tokens: row
+  // m holds basis m % 32 (m % 64 at ranks above 32; zero past r), 64 tokens = 128
+  // bytes, 16-byte piece c of row m at piece c ^ (m & 7).
+  for (int e = threadIdx.x; e < kParts * M * 8; e += kThreads) {
+    const int part = e / (M * 8), m = (e >> 3) % M, c = e & 7;
     const int q = m & (HI ? 63 : 31);
     uint32_t w[4];
 #pragma unroll
     for (int h = 0; h < 4; ++h) {
-      const int tok = c * 8 + 2 * h;
+      const int tok = part * 64 + c * 8 + 2 * h;
       w[h] = basis_bits<K>(mp, q, p.r, tok) | (basis_bits<K>(mp, q, p.r, tok + 1) << 16);
     }
-    *reinterpret_cast<uint4*>(sA + m * 128 + ((c ^ (m & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+    *reinterpret_cast<uint4*>(sA + part * kPanelBytes + m * 128 + ((c ^ (m & 7)) << 4)) =
+        make_uint4(w[0], w[1], w[2], w[3]);
   }
   ptx::fence_proxy_async_smem();   // the tensor core reads A through the async proxy
   if (warp == 4) {
@@ -230,23 +241,29 @@ __global__ void __launch_bounds__(kThreads, 1)
       Cursor c;
       if (my_quads > 0) c.decode(p, blockIdx.x);
       bool ok = true;
-      for (uint32_t n = 0; n < my_quads && !p.test_stall; ++n) {
-        const int s = static_cast<int>(n % kStages);
-        if (!ptx::mbar_wait(&empty_bar[s], ((n / kStages) + 1) & 1u, p.status, (6u << 16) | 1u)) {
-          ok = false;
-          break;
-        }
+      uint32_t it = 0;   // stages issued so far
+      for (uint32_t n = 0; n < my_quads && !p.test_stall && ok; ++n) {
         const int chunk = static_cast<int>(c.chunk) * kQuad + warp;
-        if (chunk * 64 < p.C[c.which]) {
-          // the whole box counts, also where it hangs over the tensor (zero fill)
-          ptx::mbar_expect_tx(&full_bar[s], kTileBytes);
-          ptx::tma_load_4d_hint(smem + s * kStageBytes + warp * kTileBytes, c.which ? &tmap1 : &tmap0,
-                                &full_bar[s], chunk * 64, static_cast<int32_t>(c.bw * K),
-                                static_cast<int32_t>(c.bh * K), static_cast<int32_t>(c.b), stream_once);
-        } else {
-          ptx::mbar_arrive(&full_bar[s]);   // no such chunk: what lies in the stage is multiplied and dropped
+        const bool have = chunk * 64 < p.C[c.which];
+        for (int part = 0; part < kParts; ++part, ++it) {
+          const int s = static_cast<int>(it % kStages);
+          if (!ptx::mbar_wait(&empty_bar[s], ((it / kStages) + 1) & 1u, p.status, (6u << 16) | 1u)) {
+            ok = false;
+            break;
+          }
+          if (have) {
+            // the whole box counts, also where it hangs over the tensor (zero fill);
+            // order 16: part = four token rows of the block
+            ptx::mbar_expect_tx(&full_bar[s], kTileBytes);
+            ptx::tma_load_4d_hint(smem + s * kStageBytes + warp * kTileBytes, c.which ? &tmap1 : &tmap0,
+                                  &full_bar[s], chunk * 64, static_cast<int32_t>(c.bw * K),
+                                  static_cast<int32_t>(c.bh * K + part * (64 / K)),
+                                  static_cast<int32_t>(c.b), stream_once);
+          } else {
+            ptx::mbar_arrive(&full_bar[s]);   // no such chunk: what lies in the stage is multiplied and dropped
+          }
         }
-        if (n + 1 < my_quads) c.advance(p, quad_stride, c.which ? st1 : st0);
+        if (ok && n + 1 < my_quads) c.advance(p, quad_stride, c.which ? st1 : st0);
       }
       if (!ok) *abort_flag = 1;
     }
@@ -256,25 +273,32 @@ __global__ void __launch_bounds__(kThreads, 1)
       const uint32_t idesc = ptx::idesc_bf16(M, kQuad * 64, false, true);
       const uint32_t a_addr = ptx::smem_u32(sA);
       bool ok = true;
+      uint32_t it = 0;   // stages consumed so far
       for (uint32_t n = 0; n < my_quads && ok; ++n) {
-        const int s = static_cast<int>(n % kStages);
         const int slot = static_cast<int>(n & 1u);
-        if (!ptx::mbar_wait(&acc_empty[slot], ((n >> 1) + 1) & 1u, p.status, (6u << 16) | 2u) ||
-            !ptx::mbar_wait(&full_bar[s], (n / kStages) & 1u, p.status, (6u << 16) | 3u)) {
+        if (!ptx::mbar_wait(&acc_empty[slot], ((n >> 1) + 1) & 1u, p.status, (6u << 16) | 2u)) {
           ok = false;
           break;
         }
-        ptx::tc_fence_after_sync();
-        const uint32_t sb = ptx::smem_u32(smem + s * kStageBytes);
+        for (int part = 0; part < kParts; ++part, ++it) {
+          const int s = static_cast<int>(it % kStages);
+          if (!ptx::mbar_wait(&full_bar[s], (it / kStages) & 1u, p.status, (6u << 16) | 3u)) {
+            ok = false;
+            break;
+          }
+          ptx::tc_fence_after_sync();
+          const uint32_t sb = ptx::smem_u32(smem + s * kStageBytes);
 #pragma unroll
-        for (int kk = 0; kk < (K * K) / 16; ++kk) {
-          // A: K-major, 16 tokens = 32 bytes further per step; B: MN-major, 16
-          // tokens = 16 rows of 128 bytes further, the four chunks 8 KB apart
-          const uint64_t da = ptx::smem_desc_sw128(a_addr + kk * 32, 16, 1024);
-          const uint64_t db = ptx::smem_desc_sw128(sb + kk * 2048, kTileBytes, 1024);
-          ptx::mma_bf16_ss(tmem_base + slot * kSlotCols, da, db, idesc, kk == 0 ? 0u : 1u);
+          for (int kk = 0; kk < 4; ++kk) {
+            // A: K-major, 16 tokens = 32 bytes further per step; B: MN-major, 16
+            // tokens = 16 rows of 128 bytes further, the four chunks 8 KB apart
+            const uint64_t da = ptx::smem_desc_sw128(a_addr + part * kPanelBytes + kk * 32, 16, 1024);
+            const uint64_t db = ptx::smem_desc_sw128(sb + kk * 2048, kTileBytes, 1024);
+            ptx::mma_bf16_ss(tmem_base + slot * kSlotCols, da, db, idesc, (part == 0 && kk == 0) ? 0u : 1u);
+          }
+          ptx::mma_commit(&empty_bar[s]);
         }
-        ptx::mma_commit(&empty_bar[s]);
+        if (!ok) break;
         ptx::mma_commit(&acc_full[slot]);
       }
       if (!ok) *abort_flag = 1;
@@ -289,7 +313,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     const Steps st0 = Cursor::steps(p, stride2, 0), st1 = Cursor::steps(p, stride2, 1);
     Cursor c;
     if (static_cast<uint32_t>(g) < my_quads) c.decode(p, blockIdx.x + g * gridDim.x);
-    uint8_t* const my_out = smem + kOffOut + (warp - 8) * kOutBytes;
+    uint8_t* const my_out = smem + Cfg<K>::kOffOut + (warp - 8) * kOutBytes;
     // rows this warp reads from its lane quarter, and the chunks it takes
     const int half = HI ? (w & 1) : 0;
     const int nrows = HI ? (half ? p.r - 32 : 32) : p.r;
@@ -373,7 +397,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 
 }  // namespace umma
 
-bool project_umma_supported(int k, int r) { return k == 8 && r <= 48; }
+bool project_umma_supported(int k, int r) { return (k == 8 || k == 16) && r <= 48; }
 
 int launch_project_umma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bfloat16* out1,
                         const ProjParams& p, const BasisPlan& bp, int sms, cudaStream_t stream) {
@@ -384,13 +408,16 @@ int launch_project_umma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bflo
     mp.nat_j[q] = q < bp.r ? bp.nat_j[q] : 0;
   }
   const bool hi = bp.r > 32;
-  auto kern = hi ? wht_project_umma_kernel<true> : wht_project_umma_kernel<false>;
-  static bool configured[2][64] = {};
+  const bool k16 = bp.k == 16;
+  auto kern = k16 ? (hi ? wht_project_umma_kernel<16, true> : wht_project_umma_kernel<16, false>)
+                  : (hi ? wht_project_umma_kernel<8, true> : wht_project_umma_kernel<8, false>);
+  const int smem_bytes = k16 ? Cfg<16>::kSmemBytes : Cfg<8>::kSmemBytes;
+  static bool configured[2][2][64] = {};
   int dev = 0;
   LBP_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64 || !configured[hi][dev]) {
-    LBP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    if (dev >= 0 && dev < 64) configured[hi][dev] = true;
+  if (dev < 0 || dev >= 64 || !configured[k16][hi][dev]) {
+    LBP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
+    if (dev >= 0 && dev < 64) configured[k16][hi][dev] = true;
   }
   // coefficient matrices as 2-D maps: a box is the rows x 64 channels of one item
   // that one warp writes (all r rows; at ranks above 32 the first 32 and the rest)
@@ -409,7 +436,7 @@ int launch_project_umma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bflo
   cudaLaunchAttribute attr[2];
   cfg.gridDim = dim3(projection_grid(want, sms, attr, &cfg.numAttrs));
   cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = stream;
   cfg.attrs = attr;
   LBP_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmaps[0], tmaps[1], tmout[0], tmout[1], tmouth[0], tmouth[1], out0,
