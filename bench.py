@@ -84,7 +84,7 @@ while time.time() < end:
         except Exception:
             pass
     print(repr(time.time()), mhz, mask, mx, flush=True)
-    time.sleep(0.0005)      # back-to-back NVML queries hold driver locks the launching process needs
+    time.sleep(0.001)       # every query costs the running kernels time (about 1.5 % of a step when issued back to back)
 """
 
 
@@ -137,7 +137,7 @@ class ClockSampler:
                     except ValueError:
                         pass
         inside = [r for r in rows if t_begin <= r[0] <= t_end]
-        how = "NVML from a child process, every 0.5-0.6 ms"
+        how = "NVML from a child process, about once a millisecond"
         if not inside and rows:     # a region shorter than one sampling period: the nearest sample
             mid = 0.5 * (t_begin + t_end)
             inside = [min(rows, key=lambda r: abs(r[0] - mid))]
