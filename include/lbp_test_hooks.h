@@ -6,6 +6,7 @@
 #ifndef LBP_TEST_HOOKS_H_
 #define LBP_TEST_HOOKS_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -42,6 +43,11 @@ int lbp_test_tile_plan(int Cin, int Cout, int G, int bpt, int k, int units, int 
  * again, so that one test process can run the same layer through the paths
  * the switches select.  Returns LBP_OK. */
 int lbp_test_reload_env(void);
+
+/* sizeof of the structs of include/lbp.h as the library was compiled (which: 0
+ * lbp_layer, 1 lbp_extras, 2 lbp_view, 3 lbp_basis; anything else: 0), so that a
+ * binding in another language can check its own declarations against them. */
+size_t lbp_test_struct_size(int which);
 
 #ifdef __cplusplus
 }

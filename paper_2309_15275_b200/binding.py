@@ -117,6 +117,8 @@ def _lib() -> C.CDLL:
         lib.lbp_test_tile_plan.restype = i32
         lib.lbp_test_reload_env.argtypes = []
         lib.lbp_test_reload_env.restype = i32
+        lib.lbp_test_struct_size.argtypes = [i32]
+        lib.lbp_test_struct_size.restype = sz
         lib.lbp_test_stall_products.argtypes = [i32]
         lib.lbp_test_stall_products.restype = i32
         lib.lbp_launch_count.argtypes = []
@@ -138,7 +140,7 @@ EXPORTED = ("lbp_select_bases", "lbp_basis_matrix", "lbp_flops", "lbp_status_str
             "lbp_phase_name", "lbp_select_lhe", "lbp_spectrum_workspace_bytes", "lbp_spectrum",
             "lbp_backward_batch", "lbp_test_stall_products",
             "lbp_test_reload_env", "lbp_workspace_bytes_ex", "lbp_backward_ex",
-            "lbp_backward_projected", "lbp_test_tile_plan")
+            "lbp_backward_projected", "lbp_test_tile_plan", "lbp_test_struct_size")
 
 
 def _check(status: int, where: str) -> None:

@@ -564,6 +564,16 @@ int lbp_test_tile_plan(int Cin, int Cout, int G, int bpt, int k, int units, int 
   return LBP_OK;
 }
 
+size_t lbp_test_struct_size(int which) {
+  switch (which) {
+    case 0: return sizeof(lbp_layer);
+    case 1: return sizeof(lbp_extras);
+    case 2: return sizeof(lbp_view);
+    case 3: return sizeof(lbp_basis);
+  }
+  return 0;
+}
+
 int lbp_test_reload_env(void) {
   reload_tune_options();
   return LBP_OK;

@@ -201,3 +201,13 @@ def test_tile_plan_covers_every_tile_once(Cin, Cout, G, bpt, units, pair):
 def test_tile_plan_without_a_table_for_very_many_tiles():
     info, lists = lbp.lbp_test_tile_plan(3072, 768, 400, 16, 8, 74, 1, 1)
     assert not info["listed"] and lists is None
+
+
+def test_binding_structs_have_the_size_the_library_was_compiled_with():
+    # a field added to include/lbp.h and not to the ctypes declarations (or the
+    # other way round) would shift every field behind it
+    from paper_2309_15275_b200 import binding as B
+    lib = B._lib()
+    for which, cls in ((0, B.Layer), (1, B.Extras), (2, B.View), (3, B.Basis)):
+        assert lib.lbp_test_struct_size(which) == ctypes.sizeof(cls), cls.__name__
+    assert lib.lbp_test_struct_size(99) == 0
