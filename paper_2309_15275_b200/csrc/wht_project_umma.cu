@@ -434,7 +434,12 @@ int launch_project_umma(const CUtensorMap* tmaps, __nv_bfloat16* out0, __nv_bflo
   const uint32_t want = p.n_items;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[2];
-  cfg.gridDim = dim3(projection_grid(want, sms, attr, &cfg.numAttrs));
+  // Alone on the chip the kernel is bound by HBM long before it runs out of SMs,
+  // and on three quarters of them it is about 5 % faster than on all (fewer
+  // requests in flight against one another); beside a products kernel the
+  // caller's launch shape says how many it gets.
+  const int sms_alone = projection_launch().max_ctas > 0 ? sms : (3 * sms + 3) / 4;
+  cfg.gridDim = dim3(projection_grid(want, sms_alone, attr, &cfg.numAttrs));
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = stream;
