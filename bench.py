@@ -54,7 +54,7 @@ def _peaks():
 # DRAM traffic per step (sum over the four layers, bytes) of the two kernels, from
 # the ncu capture summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum);
 # None = not captured for the current kernels.
-NCU_TRAFFIC_PER_STEP = {"wht_project_umma_kernel": 824.0e6, "lbp_products_pair_kernel": 300.0e6}
+NCU_TRAFFIC_PER_STEP = {"wht_project_umma_kernel": 824.0e6, "lbp_products_pair_kernel": 300.4e6}
 
 
 # ------------------------------------------------------------------ clocks ----
