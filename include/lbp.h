@@ -326,7 +326,7 @@ long long lbp_launch_count(void);
  * device time of phase i of Algorithm 1:
  *   1 project x and g_y (one launch)   2 (unused, recorded with 1)
  *   3 g_W product   4 g_x_hat product   5 expand
- * Where one kernel covers several phases (bf16, k = 8, r <= 16: both products
+ * Where one kernel covers several phases (bf16 on the persistent path: both products
  * and the expansion) its time shows up in the first of them and the others are
  * recorded right behind it; the full-rank mode records 0, 3 and 4 only.  lbp_phase_count() is the
  * number of events a call may record, lbp_phase_name(i) a short label. */

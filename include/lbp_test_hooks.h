@@ -14,7 +14,7 @@ extern "C" {
 #endif
 
 /* Failure injection for the bounded waits of the persistent products kernel
- * (bf16, r <= 16 path of lbp_backward).  While switched on (per calling
+ * (bf16 low-rank path of lbp_backward).  While switched on (per calling
  * thread), the TMA producer of every products launch issues no load at all.
  * Nothing is then in flight, the tensor-core issuer and the epilogue warps run
  * into their wait limits (about a second), the kernel reports LBP_ERR_TIMEOUT
