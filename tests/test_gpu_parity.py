@@ -214,6 +214,11 @@ def test_config3_through_the_switched_paths(dev, switch):
     try:
         for idx in (1, 2):
             _check_lowrank(dev, synth.config_cases(3)[idx], 8)
+        if switch == "LBP_PROJECT_UMMA":
+            # the warp-level kernels at the ranks and orders the tcgen05 kernel takes by default
+            _check_lowrank(dev, synth.config_cases(5)[1], 36, batch=2)
+            _check_lowrank(dev, synth.config_cases(5)[2], 36, batch=2)
+            _check_lowrank(dev, synth.config_cases(5)[2], 21, batch=2)
     finally:
         del os.environ[switch]
         lbp.lbp_test_reload_env()
